@@ -1,0 +1,157 @@
+/*
+ * CPU checker for batched replica placement -- TEST INFRASTRUCTURE ONLY.
+ *
+ * This file is the slow, plain definition of what the placement path computes.
+ * It exists so that tests and the benchmark's CPU-baseline leg have something
+ * independent to compare the CUDA library with. It shares no code, header,
+ * table or constant with the CUDA library, and the library never calls it.
+ *
+ * What it computes (NotebookOS, arXiv 2503.20591):
+ *
+ *   Section 3.2.1  The scheduler walks over all servers; a server that has enough
+ *                  capacity for the resource request (millicpus, memory MB, GPUs,
+ *                  VRAM GB) is a candidate. Three candidates are needed, one per
+ *                  replica. With more than three, a policy ranks them. With fewer,
+ *                  the caller has to scale out, so the count found is reported.
+ *   Section 3.4.1  Default policy. First: more idle GPUs is better. Second: the
+ *                  subscription ratio SR = S / (G * R), S = subscribed GPUs,
+ *                  G = GPUs of the server, R = replicas per kernel. A server is
+ *                  rejected if adding the replica would push its SR above the
+ *                  limit.
+ *   Section 3.2.3  A migration target additionally needs enough idle GPUs to bind
+ *                  them at once (flag NBOS_ORACLE_REQUIRE_IDLE_GPUS).
+ *
+ * Readings where the paper is silent (the project's design notes list them all):
+ *   - "idle GPUs" of a server is G - C, C = GPUs bound to running replicas.
+ *   - the SR used for ranking and for the limit is the one AFTER placement,
+ *     (S + g) / (G * R); lower is better; "exceed" means strictly greater.
+ *   - remaining ties go to the lower host index.
+ *   - a request with a negative field fits nowhere; a server with G < 1 is not a
+ *     GPU server and is never a candidate.
+ *   - every request of a batch sees the same frozen snapshot.
+ *
+ * All ratio comparisons are exact: 64-bit cross-multiplication, never floating
+ * point, never a packed key. One thread, no blocking, no early exit.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+
+#define NBOS_ORACLE_KEY_IDLE_FIRST 0 /* Section 3.4.1 order: idle GPUs, then SR   */
+#define NBOS_ORACLE_KEY_SR_FIRST 1   /* the two ranking fields swapped            */
+#define NBOS_ORACLE_REQUIRE_IDLE_GPUS 1
+
+#define NBOS_ORACLE_REPLICAS_PLACED 3 /* Section 3.2.1: three candidate servers */
+
+typedef struct {
+    int32_t n_hosts;
+    int32_t replicas_R;
+    int32_t key_order;
+    int32_t flags;
+    int64_t limit_num, limit_den; /* SR limit = limit_num / limit_den, limit_den > 0 */
+    const int32_t *G, *S, *C;     /* [n_hosts] total / subscribed / committed GPUs  */
+    const int32_t *AV, *AC, *AM;  /* [n_hosts] VRAM GB / millicpus / memory MB capacity */
+} nbos_oracle_cluster;
+
+/* SR = S / (G * R), Section 3.4.1. Only used to pin the paper's printed example. */
+double nbos_oracle_subscription_ratio(int64_t S, int64_t G, int64_t R)
+{
+    return (double)S / ((double)G * (double)R);
+}
+
+/* Sign of (Sa + g) / (Ga * R) - (Sb + g) / (Gb * R), exactly. Ga, Gb, R >= 1. */
+int nbos_oracle_compare_sr_after(int64_t Sa, int64_t Ga, int64_t Sb, int64_t Gb, int64_t g,
+                                 int64_t R)
+{
+    int64_t lhs = (Sa + g) * (Gb * R);
+    int64_t rhs = (Sb + g) * (Ga * R);
+    return (lhs > rhs) - (lhs < rhs);
+}
+
+/* Is server h a candidate for the request (g, v, c, m)? Sections 3.2.1, 3.4.1, 3.2.3. */
+int nbos_oracle_feasible(const nbos_oracle_cluster *cl, int32_t h, int32_t g, int32_t v, int32_t c,
+                         int32_t m)
+{
+    int64_t G = cl->G[h], S = cl->S[h], C = cl->C[h], R = cl->replicas_R;
+    if (g < 0 || v < 0 || c < 0 || m < 0) return 0;
+    if (G < 1) return 0;
+    /* enough capacity in each of the four resources (Section 3.2.1) */
+    if (g > G) return 0;
+    if (v > cl->AV[h]) return 0;
+    if (c > cl->AC[h]) return 0;
+    if (m > cl->AM[h]) return 0;
+    /* SR after placement must not exceed the limit (Section 3.4.1):
+     *   (S + g) / (G * R) <= num / den   <=>   (S + g) * den <= num * G * R   */
+    if ((S + (int64_t)g) * cl->limit_den > cl->limit_num * G * R) return 0;
+    /* migration reading (Section 3.2.3): the GPUs must be idle right now */
+    if ((cl->flags & NBOS_ORACLE_REQUIRE_IDLE_GPUS) && (int64_t)g > G - C) return 0;
+    return 1;
+}
+
+/* Does candidate a rank strictly before candidate b for a request of g GPUs? */
+int nbos_oracle_ranks_before(const nbos_oracle_cluster *cl, int32_t a, int32_t b, int32_t g)
+{
+    int64_t idle_a = (int64_t)cl->G[a] - cl->C[a];
+    int64_t idle_b = (int64_t)cl->G[b] - cl->C[b];
+    int sr = nbos_oracle_compare_sr_after(cl->S[a], cl->G[a], cl->S[b], cl->G[b], g,
+                                          cl->replicas_R);
+    if (cl->key_order == NBOS_ORACLE_KEY_SR_FIRST) {
+        if (sr != 0) return sr < 0;             /* lower SR first            */
+        if (idle_a != idle_b) return idle_a > idle_b; /* then more idle GPUs */
+    } else {
+        if (idle_a != idle_b) return idle_a > idle_b; /* more idle GPUs first */
+        if (sr != 0) return sr < 0;             /* then lower SR             */
+    }
+    return a < b; /* then lower host index */
+}
+
+/*
+ * Place `batch` requests against one snapshot.
+ *   requests  [batch][4] = (GPUs, VRAM GB, millicpus, memory MB)
+ *   out_hosts [batch][3] best first, -1 where fewer than three servers fit
+ *   out_found [batch]    number of servers found, 0..3 (may be NULL)
+ * Returns 0, or -1 on a bad argument / allocation failure.
+ */
+int nbos_oracle_place(const nbos_oracle_cluster *cl, const int32_t *requests, int64_t batch,
+                      int32_t *out_hosts, int32_t *out_found)
+{
+    if (!cl || cl->n_hosts < 0 || cl->limit_den <= 0 || cl->limit_num < 0 || cl->replicas_R < 1 ||
+        batch < 0)
+        return -1;
+    int32_t H = cl->n_hosts;
+    int32_t *cand = (int32_t *)malloc(sizeof(int32_t) * (size_t)(H > 0 ? H : 1));
+    char *taken = (char *)malloc((size_t)(H > 0 ? H : 1));
+    if (!cand || !taken) {
+        free(cand);
+        free(taken);
+        return -1;
+    }
+    for (int64_t r = 0; r < batch; ++r) {
+        int32_t g = requests[4 * r + 0], v = requests[4 * r + 1];
+        int32_t c = requests[4 * r + 2], m = requests[4 * r + 3];
+        /* 1. collect every candidate */
+        int32_t n_cand = 0;
+        for (int32_t h = 0; h < H; ++h)
+            if (nbos_oracle_feasible(cl, h, g, v, c, m)) cand[n_cand++] = h;
+        for (int32_t i = 0; i < n_cand; ++i) taken[i] = 0;
+        /* 2. three times: take the best candidate not taken yet */
+        int32_t found = 0;
+        for (int k = 0; k < NBOS_ORACLE_REPLICAS_PLACED; ++k) {
+            int32_t best = -1;
+            for (int32_t i = 0; i < n_cand; ++i) {
+                if (taken[i]) continue;
+                if (best < 0 || nbos_oracle_ranks_before(cl, cand[i], cand[best], g)) best = i;
+            }
+            if (best >= 0) {
+                taken[best] = 1;
+                out_hosts[3 * r + k] = cand[best];
+                ++found;
+            } else {
+                out_hosts[3 * r + k] = -1;
+            }
+        }
+        if (out_found) out_found[r] = found;
+    }
+    free(cand);
+    free(taken);
+    return 0;
+}
