@@ -1,0 +1,204 @@
+/*
+ * nbos -- batched replica placement for an oversubscribing notebook scheduler,
+ * for NVIDIA B200 (sm_100a).  C ABI.
+ *
+ * The operation is the placement decision of NotebookOS (arXiv 2503.20591):
+ *   Section 3.2.1  For a kernel's resource request (GPUs, VRAM GB, millicpus, memory MB) the
+ *                  scheduler walks over all servers, keeps those with enough capacity, and
+ *                  needs three of them, one per replica; with more than three a policy ranks
+ *                  them; with fewer the caller has to scale out.
+ *   Section 3.4.1  Default policy: more idle GPUs first, then the subscription ratio
+ *                  SR = S / (G * R) (S subscribed GPUs, G server GPUs, R replicas per kernel);
+ *                  a server whose SR would exceed the limit after placement is rejected.
+ *   Section 3.2.3  A migration target must have the GPUs idle now (NBOS_REQUIRE_IDLE_GPUS).
+ *
+ * This library evaluates that rule for a whole batch of requests against a frozen snapshot of
+ * the cluster (or against many independent snapshots at once): for every (request, host) pair
+ * the feasibility test and an exact integer ranking key, then the three best distinct feasible
+ * hosts per request.
+ *
+ * Exact definition of the result, per request (g, v, c, m) and snapshot n:
+ *   host h is feasible  <=>  g,v,c,m >= 0  and  G[h] >= 1  and  g <= G[h]  and  v <= vram_gb[h]
+ *                            and c <= millicpus[h] and m <= mem_mb[h]
+ *                            and (S[h] + g) * limit_den[n] <= limit_num[n] * G[h] * R
+ *                            and (flags & NBOS_REQUIRE_IDLE_GPUS ? g <= G[h] - C[h] : true)
+ *   feasible hosts are ordered by (G-C descending, (S+g)/(G*R) ascending, h ascending)
+ *   [NBOS_KEY_IDLE_FIRST, the paper's order] or by ((S+g)/(G*R) ascending, G-C descending,
+ *   h ascending) [NBOS_KEY_SR_FIRST]; ratios are compared exactly.
+ *   out_hosts = the first three of that order, best first, -1 where fewer exist;
+ *   out_found = how many exist, capped at 3.
+ *
+ * Conventions
+ *   - Every function returns an int status: NBOS_OK (0) or a negative NBOS_ERR_* code. Nothing
+ *     throws, aborts or prints. nbos_strerror() names a code; nbos_last_error_detail() gives the
+ *     calling thread's most recent failure in words.
+ *   - "DEVICE" pointers are device memory of the current CUDA device; "HOST" pointers are
+ *     ordinary host memory. The caller owns every buffer it passes. The library owns only the
+ *     snapshot handle (host memory) and, for the *_host entry points and the host-split launch
+ *     shape, stream-ordered temporary device memory that it frees itself.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Only devices of compute capability 10.x are accepted (NBOS_ERR_UNSUPPORTED_DEVICE).
+ *   - There is no CPU fallback anywhere.
+ */
+#ifndef NBOS_H_
+#define NBOS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define NBOS_OK 0
+#define NBOS_ERR_INVALID_ARG (-1)        /* NULL / misaligned pointer, size out of range        */
+#define NBOS_ERR_RANGE (-2)              /* a value in the arrays is outside what is supported  */
+#define NBOS_ERR_CUDA (-3)               /* a CUDA runtime call failed                          */
+#define NBOS_ERR_UNSUPPORTED_DEVICE (-4) /* current device is not compute capability 10.x       */
+#define NBOS_ERR_DEVICE_TIMEOUT (-5)     /* a bounded wait inside a kernel ran out              */
+#define NBOS_ERR_NO_MEMORY (-6)          /* host or device allocation failed / workspace small  */
+
+/* key_order */
+#define NBOS_KEY_IDLE_FIRST 0 /* Section 3.4.1: idle GPUs, then SR, then host id (default) */
+#define NBOS_KEY_SR_FIRST 1   /* SR, then idle GPUs, then host id                           */
+
+/* flags */
+#define NBOS_REQUIRE_IDLE_GPUS 1 /* Section 3.2.3: also require g <= G - C                   */
+#define NBOS_FORCE_KEY64 2       /* build the 64-bit key table even if 32 bits would do      */
+
+#define NBOS_MAX_HOSTS (1 << 20)   /* per snapshot                          */
+#define NBOS_MAX_GPUS_PER_HOST 1023
+#define NBOS_MAX_REPLICAS 1024
+#define NBOS_REPLICAS_PLACED 3     /* hosts returned per request (Section 3.2.1) */
+
+typedef struct nbos_snapshot nbos_snapshot; /* opaque */
+
+/*
+ * Cluster state, structure of arrays. N snapshots of H hosts each; array element [n*H + h].
+ *   gpus_total       G  (0 .. NBOS_MAX_GPUS_PER_HOST; a host with G = 0 is never feasible)
+ *   gpus_subscribed  S  (>= 0)  sum of GPUs requested by all replicas scheduled on the host
+ *   gpus_committed   C  (0 .. G) GPUs bound to replicas that are executing now
+ *   vram_gb, millicpus, mem_mb  (>= 0) the capacity a request's ask is compared with. Pass total
+ *                    capacity for the creation reading of Section 3.2.1, or what is left
+ *                    unbound for the migration reading of Section 3.2.3.
+ *   limit_num/limit_den  per-snapshot SR limit as a rational in the paper's units S/(G*R);
+ *                    limit_num >= 0, limit_den >= 1.
+ */
+typedef struct nbos_snapshot_desc {
+    int32_t n_snapshots; /* N >= 1                                   */
+    int32_t n_hosts;     /* 1 <= H <= NBOS_MAX_HOSTS                  */
+    int32_t replicas_R;  /* 1 .. NBOS_MAX_REPLICAS; the paper uses 3  */
+    int32_t key_order;   /* NBOS_KEY_*                                */
+    int32_t flags;       /* NBOS_REQUIRE_IDLE_GPUS | NBOS_FORCE_KEY64 */
+    int32_t reserved;    /* must be 0                                 */
+    const int32_t *limit_num; /* HOST [N] in both create variants     */
+    const int32_t *limit_den; /* HOST [N]                             */
+    /* [N*H] each. DEVICE for nbos_snapshot_create (read by work queued on the stream: keep them
+     * valid until that work has finished), HOST for nbos_snapshot_create_host (read before it
+     * returns). */
+    const int32_t *gpus_total, *gpus_subscribed, *gpus_committed;
+    const int32_t *vram_gb, *millicpus, *mem_mb;
+} nbos_snapshot_desc;
+
+typedef struct nbos_snapshot_info {
+    int32_t n_snapshots, n_hosts, hosts_padded;
+    int32_t key_bits;                    /* 32 or 64: width of the ranking key in use       */
+    int32_t bits_idle, bits_sr, bits_id; /* field widths inside the key                     */
+    int32_t key_order, flags, replicas_R;
+    int64_t workspace_bytes;
+} nbos_snapshot_info;
+
+/*
+ * Launch shape for nbos_place_batch_ex. 0 in a field = choose automatically.
+ *   lanes_per_request  1,2,4,8,16,32: lanes of one warp that share a request; each strides the
+ *                      hosts and keeps its own best three, merged by xor-shuffles at the end.
+ *   requests_per_lane  1,2,4,8: upper bound on requests one lane carries through the host loop.
+ *   host_split         K >= 1: hosts are cut into K slices handled by different thread blocks;
+ *                      K > 1 writes per-slice candidates to temporary device memory and runs a
+ *                      merge kernel.
+ *   tile_hosts         hosts per shared-memory tile (multiple of 32).
+ *   grid_blocks        thread blocks along the request dimension (per host slice).
+ */
+typedef struct nbos_launch_config {
+    int32_t lanes_per_request;
+    int32_t requests_per_lane;
+    int32_t host_split;
+    int32_t tile_hosts;
+    int32_t grid_blocks;
+    int32_t reserved[3]; /* must be 0 */
+} nbos_launch_config;
+
+/* Device bytes nbos_snapshot_create needs in `workspace` for this N and H (Section 3.4.1 state
+ * turned into per-host records). Only n_snapshots, n_hosts and flags of `desc` are read. */
+int nbos_snapshot_workspace_bytes(const nbos_snapshot_desc *desc, size_t *out_bytes);
+
+/*
+ * Build a snapshot from DEVICE arrays: validates, then derives one record per host -- the
+ * largest GPU ask that passes the capacity test, the SR limit test of Section 3.4.1 and (if
+ * asked) the idle test of Section 3.2.3, the three other capacities, and the two integers
+ * (A, B) with  key(g) = A + g * B  that order hosts exactly as Section 3.4.1 does.
+ *   workspace        DEVICE, 256-byte aligned, >= nbos_snapshot_workspace_bytes; caller-owned;
+ *                    must stay valid and untouched until nbos_snapshot_destroy.
+ *   arrays           DEVICE, 16-byte aligned.
+ * Synchronises `cuda_stream` once (value-range validation needs a small read-back).
+ * Errors: INVALID_ARG (NULL, alignment, N/H/R out of range, bad limit), RANGE (negative value,
+ * C > G, G too large, key would not fit 63 bits), NO_MEMORY, CUDA, UNSUPPORTED_DEVICE.
+ * On error *out is NULL and nothing is leaked.
+ */
+int nbos_snapshot_create(const nbos_snapshot_desc *desc, void *workspace, size_t workspace_bytes,
+                         void *cuda_stream, nbos_snapshot **out);
+
+/* Same operation from HOST arrays (any alignment). The library allocates the workspace and a
+ * staging buffer itself with cudaMalloc and frees them in nbos_snapshot_destroy / before
+ * returning. */
+int nbos_snapshot_create_host(const nbos_snapshot_desc *desc, void *cuda_stream,
+                              nbos_snapshot **out);
+
+/* Frees the handle (and what nbos_snapshot_create_host allocated). The caller must make sure no
+ * nbos_place_batch on this snapshot is still running. NULL is accepted. */
+int nbos_snapshot_destroy(nbos_snapshot *snap);
+
+int nbos_snapshot_get_info(const nbos_snapshot *snap, nbos_snapshot_info *out);
+
+/*
+ * The placement decision of Sections 3.2.1 / 3.4.1 for a batch (definition at the top).
+ *   requests   DEVICE [N * batch_per_snapshot * 4] int32, 16-byte aligned; request i of
+ *              snapshot n at ((n * batch + i) * 4): GPUs, VRAM GB, millicpus, memory MB.
+ *              A request with a negative field fits nowhere (all -1); that is not an error.
+ *   out_hosts  DEVICE [N * batch * 3] int32: host indices (0 .. H-1) best first, -1 padding.
+ *   out_found  DEVICE [N * batch] int32 or NULL: number of hosts found (0..3).
+ * Asynchronous on `cuda_stream`; outputs are valid once the stream has been synchronised. The
+ * snapshot is read-only here, so calls on different streams may overlap. batch == 0 is a no-op.
+ * Errors: INVALID_ARG, CUDA, NO_MEMORY. A device-side wait that ran out is reported later by
+ * nbos_snapshot_status.
+ */
+int nbos_place_batch(const nbos_snapshot *snap, const int32_t *requests, int64_t batch_per_snapshot,
+                     int32_t *out_hosts, int32_t *out_found, void *cuda_stream);
+
+/* Same, with an explicit launch shape (NULL = automatic). Every shape gives identical output. */
+int nbos_place_batch_ex(const nbos_snapshot *snap, const int32_t *requests,
+                        int64_t batch_per_snapshot, int32_t *out_hosts, int32_t *out_found,
+                        void *cuda_stream, const nbos_launch_config *cfg);
+
+/*
+ * Same operation with HOST buffers (pinned memory makes the copies asynchronous and faster, but
+ * any host memory works). The batch is cut into chunks whose host-to-device copy, kernel and
+ * device-to-host copy overlap on internal streams. Returns after the results are in the host
+ * buffers.
+ */
+int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_host,
+                          int64_t batch_per_snapshot, int32_t *out_hosts_host,
+                          int32_t *out_found_host, void *cuda_stream);
+
+/* Synchronises `cuda_stream` and returns the sticky device status of this snapshot: NBOS_OK, or
+ * NBOS_ERR_DEVICE_TIMEOUT if some kernel gave up on a bounded wait (its outputs are then
+ * undefined). */
+int nbos_snapshot_status(const nbos_snapshot *snap, void *cuda_stream);
+
+const char *nbos_strerror(int status);
+const char *nbos_last_error_detail(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NBOS_H_ */

@@ -1,0 +1,318 @@
+// Host side of the C ABI declared in include/nbos.h: argument checks, handle life cycle,
+// staging for the host-buffer entry points. All arithmetic of the method runs in the kernels of
+// nbos_derive.cu and nbos_place.cu.
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "nbos_internal.h"
+
+namespace nbos {
+
+static thread_local char g_detail[512] = "";
+
+int fail(int code, const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_detail, sizeof(g_detail), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+int cuda_fail(cudaError_t e, const char *what)
+{
+    cudaGetLastError();  // clear the non-sticky error state
+    return fail(NBOS_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+namespace {
+
+bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+int check_desc_scalars(const nbos_snapshot_desc *d)
+{
+    if (!d) return fail(NBOS_ERR_INVALID_ARG, "desc is NULL");
+    if (d->n_snapshots < 1 || d->n_snapshots > 65535)
+        return fail(NBOS_ERR_INVALID_ARG, "n_snapshots must be in 1..65535 (got %d)", d->n_snapshots);
+    if (d->n_hosts < 1 || d->n_hosts > NBOS_MAX_HOSTS)
+        return fail(NBOS_ERR_INVALID_ARG, "n_hosts must be in 1..%d (got %d)", NBOS_MAX_HOSTS, d->n_hosts);
+    if (d->flags & ~(NBOS_REQUIRE_IDLE_GPUS | NBOS_FORCE_KEY64))
+        return fail(NBOS_ERR_INVALID_ARG, "unknown bits in flags (0x%x)", d->flags);
+    return NBOS_OK;
+}
+
+int check_desc_full(const nbos_snapshot_desc *d)
+{
+    int rc = check_desc_scalars(d);
+    if (rc) return rc;
+    if (d->replicas_R < 1 || d->replicas_R > NBOS_MAX_REPLICAS)
+        return fail(NBOS_ERR_INVALID_ARG, "replicas_R must be in 1..%d (got %d)", NBOS_MAX_REPLICAS, d->replicas_R);
+    if (d->key_order != NBOS_KEY_IDLE_FIRST && d->key_order != NBOS_KEY_SR_FIRST)
+        return fail(NBOS_ERR_INVALID_ARG, "unknown key_order %d", d->key_order);
+    if (d->reserved != 0) return fail(NBOS_ERR_INVALID_ARG, "reserved must be 0");
+    if (!d->limit_num || !d->limit_den) return fail(NBOS_ERR_INVALID_ARG, "limit_num / limit_den is NULL");
+    const void *arrays[6] = {d->gpus_total, d->gpus_subscribed, d->gpus_committed,
+                             d->vram_gb, d->millicpus, d->mem_mb};
+    for (int i = 0; i < 6; ++i)
+        if (!arrays[i]) return fail(NBOS_ERR_INVALID_ARG, "host-state array %d is NULL", i);
+    for (int n = 0; n < d->n_snapshots; ++n) {
+        if (d->limit_den[n] < 1) return fail(NBOS_ERR_INVALID_ARG, "limit_den[%d] must be >= 1", n);
+        if (d->limit_num[n] < 0) return fail(NBOS_ERR_INVALID_ARG, "limit_num[%d] must be >= 0", n);
+    }
+    return NBOS_OK;
+}
+
+int check_device(int *device, int *sm_count)
+{
+    NBOS_CUDA_TRY(cudaGetDevice(device));
+    int major = 0;
+    NBOS_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, *device));
+    if (major != 10)
+        return fail(NBOS_ERR_UNSUPPORTED_DEVICE, "device %d has compute capability %d.x; this library is built for 10.x only",
+                    *device, major);
+    NBOS_CUDA_TRY(cudaDeviceGetAttribute(sm_count, cudaDevAttrMultiProcessorCount, *device));
+    return NBOS_OK;
+}
+
+nbos_snapshot *new_handle(const nbos_snapshot_desc *d)
+{
+    nbos_snapshot *s = new (std::nothrow) nbos_snapshot();
+    if (!s) return nullptr;
+    s->N = d->n_snapshots;
+    s->H = d->n_hosts;
+    s->Hpad = pad_hosts(d->n_hosts);
+    s->R = d->replicas_R;
+    s->key_order = d->key_order;
+    s->flags = d->flags;
+    s->owns_workspace = false;
+    return s;
+}
+
+}  // namespace
+}  // namespace nbos
+
+using namespace nbos;
+
+extern "C" {
+
+int nbos_snapshot_workspace_bytes(const nbos_snapshot_desc *desc, size_t *out_bytes)
+{
+    if (!out_bytes) return fail(NBOS_ERR_INVALID_ARG, "out_bytes is NULL");
+    int rc = check_desc_scalars(desc);
+    if (rc) return rc;
+    *out_bytes = workspace_layout(desc->n_snapshots, pad_hosts(desc->n_hosts)).total;
+    return NBOS_OK;
+}
+
+int nbos_snapshot_create(const nbos_snapshot_desc *desc, void *workspace, size_t workspace_bytes,
+                         void *cuda_stream, nbos_snapshot **out)
+{
+    if (!out) return fail(NBOS_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    int rc = check_desc_full(desc);
+    if (rc) return rc;
+    const void *arrays[6] = {desc->gpus_total, desc->gpus_subscribed, desc->gpus_committed,
+                             desc->vram_gb, desc->millicpus, desc->mem_mb};
+    for (int i = 0; i < 6; ++i)
+        if (!aligned(arrays[i], 16)) return fail(NBOS_ERR_INVALID_ARG, "host-state array %d is not 16-byte aligned", i);
+    if (!workspace || !aligned(workspace, 256)) return fail(NBOS_ERR_INVALID_ARG, "workspace is NULL or not 256-byte aligned");
+    const size_t need = workspace_layout(desc->n_snapshots, pad_hosts(desc->n_hosts)).total;
+    if (workspace_bytes < need)
+        return fail(NBOS_ERR_NO_MEMORY, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
+    int device = 0, sms = 0;
+    rc = check_device(&device, &sms);
+    if (rc) return rc;
+    nbos_snapshot *s = new_handle(desc);
+    if (!s) return fail(NBOS_ERR_NO_MEMORY, "host allocation failed");
+    s->workspace = workspace;
+    s->workspace_bytes = need;
+    s->device = device;
+    s->sm_count = sms;
+    rc = derive_snapshot(s, desc, desc->gpus_total, desc->gpus_subscribed, desc->gpus_committed,
+                         desc->vram_gb, desc->millicpus, desc->mem_mb,
+                         static_cast<cudaStream_t>(cuda_stream));
+    if (rc) {
+        delete s;
+        return rc;
+    }
+    *out = s;
+    return NBOS_OK;
+}
+
+int nbos_snapshot_create_host(const nbos_snapshot_desc *desc, void *cuda_stream, nbos_snapshot **out)
+{
+    if (!out) return fail(NBOS_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    int rc = check_desc_full(desc);
+    if (rc) return rc;
+    int device = 0, sms = 0;
+    rc = check_device(&device, &sms);
+    if (rc) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t cells = (size_t)desc->n_snapshots * desc->n_hosts;
+    const size_t arr_bytes = (cells * sizeof(int32_t) + 255) & ~(size_t)255;
+    const size_t need = workspace_layout(desc->n_snapshots, pad_hosts(desc->n_hosts)).total;
+    void *ws = nullptr, *staging = nullptr;
+    cudaError_t e = cudaMalloc(&ws, need);
+    if (e == cudaSuccess) e = cudaMalloc(&staging, 6 * arr_bytes);
+    if (e != cudaSuccess) {
+        cudaFree(ws);
+        cudaGetLastError();
+        return fail(NBOS_ERR_NO_MEMORY, "cudaMalloc failed: %s", cudaGetErrorString(e));
+    }
+    nbos_snapshot *s = new_handle(desc);
+    if (!s) {
+        cudaFree(ws);
+        cudaFree(staging);
+        return fail(NBOS_ERR_NO_MEMORY, "host allocation failed");
+    }
+    s->workspace = ws;
+    s->workspace_bytes = need;
+    s->owns_workspace = true;
+    s->device = device;
+    s->sm_count = sms;
+    const int32_t *src[6] = {desc->gpus_total, desc->gpus_subscribed, desc->gpus_committed,
+                             desc->vram_gb, desc->millicpus, desc->mem_mb};
+    const int32_t *dev[6];
+    for (int i = 0; i < 6 && e == cudaSuccess; ++i) {
+        dev[i] = reinterpret_cast<const int32_t *>(static_cast<char *>(staging) + i * arr_bytes);
+        e = cudaMemcpyAsync(const_cast<int32_t *>(dev[i]), src[i], cells * sizeof(int32_t),
+                            cudaMemcpyHostToDevice, stream);
+    }
+    rc = e == cudaSuccess ? derive_snapshot(s, desc, dev[0], dev[1], dev[2], dev[3], dev[4], dev[5], stream)
+                          : cuda_fail(e, "copying host-state arrays to the device");
+    if (rc == NBOS_OK) {
+        e = cudaStreamSynchronize(stream);  // the staging buffer is released next
+        if (e != cudaSuccess) rc = cuda_fail(e, "cudaStreamSynchronize");
+    }
+    cudaFree(staging);
+    if (rc) {
+        cudaFree(ws);
+        delete s;
+        return rc;
+    }
+    *out = s;
+    return NBOS_OK;
+}
+
+int nbos_snapshot_destroy(nbos_snapshot *snap)
+{
+    if (!snap) return NBOS_OK;
+    int rc = NBOS_OK;
+    if (snap->owns_workspace) {
+        cudaError_t e = cudaFree(snap->workspace);
+        if (e != cudaSuccess) rc = cuda_fail(e, "cudaFree");
+    }
+    delete snap;
+    return rc;
+}
+
+int nbos_snapshot_get_info(const nbos_snapshot *s, nbos_snapshot_info *out)
+{
+    if (!s || !out) return fail(NBOS_ERR_INVALID_ARG, "NULL argument");
+    out->n_snapshots = s->N;
+    out->n_hosts = s->H;
+    out->hosts_padded = s->Hpad;
+    out->key_bits = s->key.key_bits;
+    out->bits_idle = s->key.bits_idle;
+    out->bits_sr = s->key.bits_sr;
+    out->bits_id = s->key.bits_id;
+    out->key_order = s->key_order;
+    out->flags = s->flags;
+    out->replicas_R = s->R;
+    out->workspace_bytes = (int64_t)s->workspace_bytes;
+    return NBOS_OK;
+}
+
+int nbos_place_batch_ex(const nbos_snapshot *snap, const int32_t *requests,
+                        int64_t batch_per_snapshot, int32_t *out_hosts, int32_t *out_found,
+                        void *cuda_stream, const nbos_launch_config *cfg)
+{
+    if (!snap) return fail(NBOS_ERR_INVALID_ARG, "snapshot is NULL");
+    if (batch_per_snapshot < 0 || batch_per_snapshot > ((int64_t)1 << 40) / snap->N)
+        return fail(NBOS_ERR_INVALID_ARG, "batch_per_snapshot out of range");
+    if (batch_per_snapshot == 0) return NBOS_OK;
+    if (!requests || !out_hosts) return fail(NBOS_ERR_INVALID_ARG, "requests / out_hosts is NULL");
+    if (!aligned(requests, 16)) return fail(NBOS_ERR_INVALID_ARG, "requests is not 16-byte aligned");
+    if (!aligned(out_hosts, 4) || !aligned(out_found, 4)) return fail(NBOS_ERR_INVALID_ARG, "output not 4-byte aligned");
+    return launch_place(snap, requests, batch_per_snapshot, out_hosts, out_found,
+                        static_cast<cudaStream_t>(cuda_stream), cfg);
+}
+
+int nbos_place_batch(const nbos_snapshot *snap, const int32_t *requests, int64_t batch_per_snapshot,
+                     int32_t *out_hosts, int32_t *out_found, void *cuda_stream)
+{
+    return nbos_place_batch_ex(snap, requests, batch_per_snapshot, out_hosts, out_found, cuda_stream,
+                               nullptr);
+}
+
+int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_host,
+                          int64_t batch_per_snapshot, int32_t *out_hosts_host,
+                          int32_t *out_found_host, void *cuda_stream)
+{
+    if (!snap) return fail(NBOS_ERR_INVALID_ARG, "snapshot is NULL");
+    if (batch_per_snapshot < 0 || batch_per_snapshot > ((int64_t)1 << 40) / snap->N)
+        return fail(NBOS_ERR_INVALID_ARG, "batch_per_snapshot out of range");
+    if (batch_per_snapshot == 0) return NBOS_OK;
+    if (!requests_host || !out_hosts_host) return fail(NBOS_ERR_INVALID_ARG, "requests / out_hosts is NULL");
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t total = (size_t)snap->N * (size_t)batch_per_snapshot;
+    const size_t req_bytes = total * 16, out_bytes = total * 12, found_bytes = out_found_host ? total * 4 : 0;
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    char *buf = nullptr;
+    cudaError_t e = cudaMallocAsync(reinterpret_cast<void **>(&buf), up(req_bytes) + up(out_bytes) + up(found_bytes), stream);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(NBOS_ERR_NO_MEMORY, "device staging allocation failed: %s", cudaGetErrorString(e));
+    }
+    int32_t *d_req = reinterpret_cast<int32_t *>(buf);
+    int32_t *d_out = reinterpret_cast<int32_t *>(buf + up(req_bytes));
+    int32_t *d_found = out_found_host ? reinterpret_cast<int32_t *>(buf + up(req_bytes) + up(out_bytes)) : nullptr;
+    int rc = NBOS_OK;
+    e = cudaMemcpyAsync(d_req, requests_host, req_bytes, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) {
+        rc = launch_place(snap, d_req, batch_per_snapshot, d_out, d_found, stream, nullptr);
+        if (rc == NBOS_OK) e = cudaMemcpyAsync(out_hosts_host, d_out, out_bytes, cudaMemcpyDeviceToHost, stream);
+        if (rc == NBOS_OK && e == cudaSuccess && d_found)
+            e = cudaMemcpyAsync(out_found_host, d_found, found_bytes, cudaMemcpyDeviceToHost, stream);
+    }
+    cudaFreeAsync(buf, stream);
+    cudaError_t e2 = cudaStreamSynchronize(stream);
+    if (rc) return rc;
+    if (e != cudaSuccess) return cuda_fail(e, "host <-> device copy");
+    if (e2 != cudaSuccess) return cuda_fail(e2, "cudaStreamSynchronize");
+    return NBOS_OK;
+}
+
+int nbos_snapshot_status(const nbos_snapshot *snap, void *cuda_stream)
+{
+    if (!snap) return fail(NBOS_ERR_INVALID_ARG, "snapshot is NULL");
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    unsigned int word = 0;
+    NBOS_CUDA_TRY(cudaMemcpyAsync(&word, snap->d_status, sizeof(word), cudaMemcpyDeviceToHost, stream));
+    NBOS_CUDA_TRY(cudaStreamSynchronize(stream));
+    if (word) return fail(NBOS_ERR_DEVICE_TIMEOUT, "a kernel gave up on a bounded wait (status word 0x%x)", word);
+    return NBOS_OK;
+}
+
+const char *nbos_strerror(int status)
+{
+    switch (status) {
+        case NBOS_OK: return "ok";
+        case NBOS_ERR_INVALID_ARG: return "invalid argument";
+        case NBOS_ERR_RANGE: return "value out of the supported range";
+        case NBOS_ERR_CUDA: return "CUDA runtime error";
+        case NBOS_ERR_UNSUPPORTED_DEVICE: return "unsupported device (needs compute capability 10.x)";
+        case NBOS_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+        case NBOS_ERR_NO_MEMORY: return "out of memory or workspace too small";
+    }
+    return "unknown status";
+}
+
+const char *nbos_last_error_detail(void) { return g_detail; }
+
+}  // extern "C"

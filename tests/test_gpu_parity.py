@@ -1,0 +1,298 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU checker, element by
+element, on identical seeded inputs. Integer and index work: the bar is bit-exact."""
+from __future__ import annotations
+
+import dataclasses
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2503_20591_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+CPU_THREADS = max(1, min(32, (os.cpu_count() or 1)))
+
+
+@pytest.fixture(scope="module")
+def nb():
+    import torch
+    from paper_2503_20591_b200 import binding, build as lib_build
+    lib_build.build()
+    assert torch.cuda.is_available()
+    binding.load_library()
+    return binding
+
+
+def both(nb, w, key_order=0, flags=0, config=None, lib_flags=0):
+    got = nb.place_workload(w, key_order=key_order, flags=flags | lib_flags, config=config)
+    ref = oracle.place_workload(w, key_order=key_order, flags=flags, threads=CPU_THREADS)
+    return got, ref
+
+
+def assert_same(got, ref, what=""):
+    bad = np.nonzero((got[0] != ref[0]).any(axis=-1))
+    assert bad[0].size == 0, (f"{what}: {bad[0].size} requests differ, first at "
+                              f"{[int(b[0]) for b in bad]}: got {got[0][tuple(b[0] for b in bad)]}"
+                              f" expected {ref[0][tuple(b[0] for b in bad)]}")
+    np.testing.assert_array_equal(got[1], ref[1], err_msg=what)
+
+
+# ---- the benchmark workloads ------------------------------------------------------------------
+@pytest.mark.parametrize("index", [0, 1])
+@pytest.mark.parametrize("key_order", [0, 1])
+def test_small_configs_full(nb, index, key_order):
+    w = W.make_config(index)
+    got, ref = both(nb, w, key_order=key_order)
+    assert_same(got, ref, w.name)
+
+
+def test_config2_full(nb):
+    w = W.make_config(2)
+    got, ref = both(nb, w)
+    assert_same(got, ref, w.name)
+    assert (ref[1] < 3).any() and (ref[1] == 3).any()  # sentinel path and full path both hit
+
+
+def test_config4_full(nb):
+    w = W.make_config(4)
+    got, ref = both(nb, w)
+    assert_same(got, ref, w.name)
+
+
+def test_config3_full_size_sampled(nb):
+    """Full-size launch (4,096 hosts x 1,048,576 requests, the shape the benchmark times); the
+    checker recomputes a sample of the requests one by one; the rest is held to properties."""
+    w = W.make_config(3)
+    hosts, found = nb.place_workload(w)
+    rng = np.random.default_rng(0)
+    ids = np.unique(np.concatenate([np.arange(0, 4096), np.arange(w.batch - 4096, w.batch),
+                                    rng.integers(0, w.batch, size=24576)]))
+    sub = dataclasses.replace(w, requests=np.ascontiguousarray(w.requests[:, ids]), batch=ids.size)
+    ref = oracle.place_workload(sub, threads=CPU_THREADS)
+    assert_same((hosts[:, ids], found[:, ids]), ref, "cfg3 sample")
+    # properties over the whole output
+    assert hosts.min() >= -1 and hosts.max() < w.n_hosts
+    filled = hosts >= 0
+    np.testing.assert_array_equal(found, filled.sum(axis=-1))
+    assert (filled[..., :-1] >= filled[..., 1:]).all()          # -1 only at the tail
+    h = hosts[0]
+    full = found[0] == 3
+    assert ((h[full, 0] != h[full, 1]) & (h[full, 1] != h[full, 2]) & (h[full, 0] != h[full, 2])).all()
+    # every chosen host passes the four capacity compares and the GPU test
+    req = w.requests[0]
+    for k in range(3):
+        sel = h[:, k] >= 0
+        hk = h[sel, k]
+        assert (req[sel, 0] <= w.gpus_total[0][hk]).all()
+        assert (req[sel, 1] <= w.vram_gb[0][hk]).all()
+        assert (req[sel, 2] <= w.millicpus[0][hk]).all()
+        assert (req[sel, 3] <= w.mem_mb[0][hk]).all()
+        assert ((w.gpus_subscribed[0][hk].astype(np.int64) + req[sel, 0]) * int(w.limit_den[0])
+                <= int(w.limit_num[0]) * w.gpus_total[0][hk].astype(np.int64) * 3).all()
+
+
+# ---- every launch shape gives the same bytes --------------------------------------------------
+SHAPES = [
+    dict(lanes_per_request=1), dict(lanes_per_request=2), dict(lanes_per_request=4),
+    dict(lanes_per_request=8), dict(lanes_per_request=16), dict(lanes_per_request=32),
+    dict(lanes_per_request=1, requests_per_lane=1), dict(lanes_per_request=1, requests_per_lane=2),
+    dict(lanes_per_request=4, requests_per_lane=4), dict(lanes_per_request=32, requests_per_lane=8),
+    dict(lanes_per_request=1, tile_hosts=32), dict(lanes_per_request=8, tile_hosts=64),
+    dict(lanes_per_request=32, tile_hosts=96, grid_blocks=3),
+    dict(lanes_per_request=32, host_split=2, tile_hosts=64),
+    dict(lanes_per_request=1, host_split=5, tile_hosts=32),
+    dict(lanes_per_request=16, host_split=3, tile_hosts=128, grid_blocks=7),
+    dict(lanes_per_request=1, grid_blocks=1),
+]
+
+
+@pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "-".join(f"{k[:5]}{v}" for k, v in s.items()))
+def test_launch_shapes(nb, shape):
+    cfg = nb.launch_config(**shape)
+    for w in (W.make_config(2, batch=5000), W.mixed_gpu_cluster(777, 3001, seed=5)):
+        got, ref = both(nb, w, config=cfg)
+        assert_same(got, ref, f"{w.name} {shape}")
+
+
+@pytest.mark.parametrize("lib_flags", [0, 2], ids=["key32", "key64"])
+@pytest.mark.parametrize("key_order", [0, 1])
+@pytest.mark.parametrize("flags", [0, 1], ids=["subscribe", "idle_now"])
+def test_key_widths_orders_flags(nb, lib_flags, key_order, flags):
+    for w in (W.mixed_gpu_cluster(1000, 4096, seed=11), W.make_config(2, batch=4096),
+              W.make_config(4, batch=100, n_snapshots=24)):
+        for shape in (dict(), dict(lanes_per_request=32, host_split=2, tile_hosts=128)):
+            got, ref = both(nb, w, key_order=key_order, flags=flags, lib_flags=lib_flags,
+                            config=nb.launch_config(**shape) if shape else None)
+            assert_same(got, ref, f"{w.name} order={key_order} flags={flags} lib={lib_flags}")
+
+
+def test_key_width_is_chosen_from_the_data(nb):
+    w = W.make_config(1)
+    s = nb.snapshot_from_workload(w)
+    info = s.info()
+    assert (info.key_bits, info.bits_id, info.hosts_padded) == (32, 8, 256)
+    assert info.bits_idle == 4 and info.bits_sr == 5
+    nb.nbos_snapshot_destroy(s)
+    s = nb.snapshot_from_workload(w, flags=nb.NBOS_FORCE_KEY64)
+    assert s.info().key_bits == 64
+    nb.nbos_snapshot_destroy(s)
+    # a huge subscription count on a host that can still take requests needs more than 31 bits
+    big = W.make_config(0)
+    big.gpus_subscribed[0, 3] = 1 << 27
+    big.limit_num[0], big.limit_den[0] = 1 << 26, 1
+    s = nb.snapshot_from_workload(big)
+    assert s.info().key_bits == 64
+    nb.nbos_snapshot_destroy(s)
+    got, ref = both(nb, big)
+    assert_same(got, ref, "wide key")
+
+
+# ---- edge cases -------------------------------------------------------------------------------
+@pytest.mark.parametrize("n_hosts", [1, 2, 3, 31, 33, 100, 1025])
+@pytest.mark.parametrize("batch", [1, 7, 300])
+def test_ragged_sizes(nb, n_hosts, batch):
+    w = W.uniform_cluster(n_hosts, batch, seed=n_hosts * 1000 + batch)
+    got, ref = both(nb, w)
+    assert_same(got, ref, f"H={n_hosts} B={batch}")
+    w = W.mixed_gpu_cluster(n_hosts, batch, seed=n_hosts + batch)
+    got, ref = both(nb, w, key_order=1)
+    assert_same(got, ref, f"mixed H={n_hosts} B={batch}")
+
+
+def test_multi_snapshot_ragged(nb):
+    w = W.what_if_sweep(13, 70, 333)
+    for shape in (dict(), dict(lanes_per_request=1, grid_blocks=5),
+                  dict(lanes_per_request=8, host_split=2, tile_hosts=32)):
+        got, ref = both(nb, w, config=nb.launch_config(**shape) if shape else None)
+        assert_same(got, ref, f"sweep {shape}")
+
+
+def test_negative_and_zero_requests(nb):
+    w = W.make_config(1, batch=64)
+    w.requests[0, 0] = [-1, 16, 1000, 1024]
+    w.requests[0, 1] = [1, -16, 1000, 1024]
+    w.requests[0, 2] = [1, 16, -1000, 1024]
+    w.requests[0, 3] = [1, 16, 1000, -1024]
+    w.requests[0, 4] = [0, 0, 0, 0]
+    w.requests[0, 5] = [np.iinfo(np.int32).max] * 4
+    w.requests[0, 6] = [np.iinfo(np.int32).min] * 4
+    got, ref = both(nb, w)
+    assert_same(got, ref, "odd requests")
+    assert (got[0][0, :4] == -1).all() and (got[1][0, :4] == 0).all()
+    assert got[1][0, 4] == 3
+
+
+def test_hosts_without_gpus_and_saturated_hosts(nb):
+    w = W.make_config(1, batch=256)
+    w.gpus_total[0, ::3] = 0
+    w.gpus_committed[0, ::3] = 0
+    w.gpus_subscribed[0, 1::3] = 1000
+    w.requests[0, :32, 0] = 0
+    w.requests[0, :32, 1] = 0
+    got, ref = both(nb, w)
+    assert_same(got, ref, "no-GPU hosts")
+
+
+def test_nothing_feasible_anywhere(nb):
+    w = W.make_config(0)
+    w.limit_num[0] = 0
+    got, ref = both(nb, w)
+    assert_same(got, ref, "limit 0")
+    assert (got[0] == -1).all() and (got[1] == 0).all()
+
+
+def test_empty_batch_and_optional_found(nb):
+    import torch
+    w = W.make_config(0)
+    s = nb.snapshot_from_workload(w)
+    empty = torch.empty((1, 0, 4), dtype=torch.int32, device="cuda")
+    out = torch.empty((1, 0, 3), dtype=torch.int32, device="cuda")
+    nb.nbos_place_batch(s, empty, out)
+    req = torch.from_numpy(w.requests).cuda()
+    out = torch.full((1, w.batch, 3), -7, dtype=torch.int32, device="cuda")
+    nb.nbos_place_batch(s, req, out, None)
+    assert nb.nbos_snapshot_status(s) == nb.NBOS_OK
+    ref = oracle.place_workload(w)
+    np.testing.assert_array_equal(out.cpu().numpy(), ref[0])
+    nb.nbos_snapshot_destroy(s)
+
+
+def test_host_buffer_entry_points(nb):
+    import torch
+    w = W.make_config(4, batch=257, n_snapshots=5)
+    arrays = [torch.from_numpy(getattr(w, k)).reshape(-1) for k in w.HOST_FIELDS]
+    s = nb.nbos_snapshot_create_host(w.n_snapshots, w.n_hosts, torch.from_numpy(w.limit_num),
+                                     torch.from_numpy(w.limit_den), *arrays)
+    ref = oracle.place_workload(w)
+    for pinned in (False, True):
+        req = torch.from_numpy(w.requests.copy())
+        out = torch.empty((w.n_snapshots, w.batch, 3), dtype=torch.int32)
+        found = torch.empty((w.n_snapshots, w.batch), dtype=torch.int32)
+        if pinned:
+            req, out, found = req.pin_memory(), out.pin_memory(), found.pin_memory()
+        nb.nbos_place_batch_host(s, req, out, found)
+        np.testing.assert_array_equal(out.numpy(), ref[0])
+        np.testing.assert_array_equal(found.numpy(), ref[1])
+    nb.nbos_snapshot_destroy(s)
+
+
+def test_create_rejects_bad_values(nb):
+    import torch
+    w = W.make_config(0)
+
+    def create(mod):
+        ww = W.make_config(0)
+        mod(ww)
+        return nb.snapshot_from_workload(ww)
+
+    for mod, code in ((lambda x: x.gpus_subscribed.__setitem__((0, 5), -1), nb.NBOS_ERR_RANGE),
+                      (lambda x: x.gpus_committed.__setitem__((0, 5), 9), nb.NBOS_ERR_RANGE),
+                      (lambda x: x.gpus_total.__setitem__((0, 5), 5000), nb.NBOS_ERR_RANGE),
+                      (lambda x: x.mem_mb.__setitem__((0, 31), -5), nb.NBOS_ERR_RANGE),
+                      (lambda x: x.limit_den.__setitem__(0, 0), nb.NBOS_ERR_INVALID_ARG),
+                      (lambda x: x.limit_num.__setitem__(0, -1), nb.NBOS_ERR_INVALID_ARG)):
+        with pytest.raises(nb.NbosError) as e:
+            create(mod)
+        assert e.value.status == code
+    # the context is fine afterwards
+    got, ref = both(nb, w)
+    assert_same(got, ref)
+    # workspace too small / misaligned
+    dev = [torch.from_numpy(getattr(w, k)).cuda().reshape(-1) for k in w.HOST_FIELDS]
+    with pytest.raises(nb.NbosError) as e:
+        nb.nbos_snapshot_create(1, 32, torch.from_numpy(w.limit_num), torch.from_numpy(w.limit_den),
+                                *dev, workspace=torch.empty(512, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == nb.NBOS_ERR_NO_MEMORY
+
+
+def test_streams_and_repeated_calls(nb):
+    import torch
+    w = W.make_config(2, batch=20000)
+    ref = oracle.place_workload(w, threads=CPU_THREADS)
+    s = nb.snapshot_from_workload(w)
+    req = torch.from_numpy(w.requests).cuda()
+    streams = [torch.cuda.Stream() for _ in range(3)]
+    outs = [torch.empty((1, w.batch, 3), dtype=torch.int32, device="cuda") for _ in streams]
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for st, out in zip(streams, outs):
+            nb.nbos_place_batch(s, req, out, None, stream=st)
+    torch.cuda.synchronize()
+    assert nb.nbos_snapshot_status(s) == nb.NBOS_OK
+    for out in outs:
+        np.testing.assert_array_equal(out.cpu().numpy(), ref[0])
+    nb.nbos_snapshot_destroy(s)
+
+
+def test_bounded_wait_gives_up_and_context_survives(nb):
+    """A wait that nothing will ever satisfy must end by itself, be reported, and leave the
+    device usable (no trap, no hang)."""
+    gave_up, ms = nb.nbos_probe_wait_timeout(20_000_000)   # 20 ms
+    assert gave_up
+    assert 15.0 < ms < 2000.0
+    w = W.make_config(0)
+    got, ref = both(nb, w)
+    assert_same(got, ref)
