@@ -1,0 +1,373 @@
+#!/usr/bin/env python
+"""Benchmark of batched replica placement on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N ...
+
+One step = the whole path on one batch: snapshot derivation from the cluster-state arrays, then
+the placement of every request of the batch (feasibility + key for every (request, host) pair,
+best three hosts per request). Default workload: 4,096 hosts x 1,048,576 requests, the largest of
+the five benchmark shapes. Prints ONE JSON line on rank 0.
+
+`--impl reference` times the plain CPU checker (as it stands, one thread) on a bounded sample of
+the same workload; it is a slow, deliberately simple program, reported for context.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+SM_COUNT_B200 = 148
+INT32_LANES_PER_SM = 64           # integer ALU lanes per SM (16 per scheduler partition)
+ALGORITHMIC_OPS_PER_PAIR = 6      # 4 capacity compares + 1 multiply-add (key) + 1 compare vs 3rd best
+L2_BYTES = 126 * 1024 * 1024
+# DRAM bytes (read + write) of one placement-kernel launch on the default workload, from the ncu
+# capture summarised under profiles/. None while no capture matches the current kernel.
+PLACE_KERNEL_DRAM_BYTES_PER_LAUNCH = None
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
+    ap.add_argument("--workload", type=int, default=3, help="benchmark workload index 0..4")
+    ap.add_argument("--batch", type=int, default=None, help="shrink the batch (profiling captures)")
+    ap.add_argument("--snapshots", type=int, default=None, help="shrink workload 4")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--cpu-sample", type=int, default=None, help="requests in the CPU sample")
+    return ap.parse_args()
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks: sampled through NVML (read-only) from a thread while the timed region runs
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {
+        0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap",
+        0x8: "hw_slowdown", 0x10: "sync_boost", 0x20: "sw_thermal_slowdown",
+        0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting",
+    }
+
+    def __init__(self, torch_device_index: int):
+        self.samples, self.reason_bits, self.power = [], 0, []
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            uuid = str(torch.cuda.get_device_properties(torch_device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except TypeError:
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:  # NVML missing: the JSON says so
+            self.error = repr(e)
+
+    def _poll(self):
+        nv, h = self._nv, self._h
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)))
+                try:
+                    self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(h))
+                except Exception:
+                    self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(h))
+                self.power.append(nv.nvmlDeviceGetPowerUsage(h) / 1000.0)
+            except Exception:
+                pass
+            time.sleep(0.004)
+
+    def start(self):
+        if self._h is not None:
+            self.samples, self.reason_bits, self.power = [], 0, []
+            self._stop.clear()
+            self._thread = threading.Thread(target=self._poll, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join()
+            self._thread = None
+
+    def summary(self):
+        if self._h is None or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [],
+                    "note": "NVML unavailable: " + getattr(self, "error", "no samples")}
+        reasons = [name for bit, name in self.REASONS.items()
+                   if self.reason_bits & bit and name != "gpu_idle"]
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": reasons, "samples": len(self.samples),
+                "power_w_max": max(self.power) if self.power else None}
+
+
+# ------------------------------------------------------------------------------------------------
+# reference arm: the CPU checker on a bounded sample
+# ------------------------------------------------------------------------------------------------
+def time_checker(w, sample: int, steps: int, warmup: int):
+    """Run the checker `warmup + steps` times over the first `sample` requests of every
+    snapshot; returns (decisions per step, seconds per step, last result)."""
+    import oracle
+    sl = slice(0, sample)
+    res = None
+    for _ in range(warmup):
+        res = oracle.place_workload(w, request_slice=sl)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        res = oracle.place_workload(w, request_slice=sl)
+    dt = (time.perf_counter() - t0) / max(1, steps)
+    return w.n_snapshots * min(sample, w.batch), dt, res
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from paper_2503_20591_b200 import workloads as W
+    w = W.make_config(args.workload, batch=args.batch, n_snapshots=args.snapshots)
+    # size the sample so that the whole run stays near a minute at ~25 M pairs/s per core
+    budget_pairs = 60.0 * 25e6 / max(1, args.steps + args.warmup)
+    sample = args.cpu_sample or int(budget_pairs / (w.n_snapshots * w.n_hosts))
+    sample = max(16, min(w.batch, 1 << max(4, sample.bit_length() - 1)))
+    dec, dt, _ = time_checker(w, sample, args.steps, args.warmup)
+    value = dec / dt
+    line = {
+        "impl": "reference", "metric": "placement decisions/sec", "value": value,
+        "unit": "decisions/s", "pairs_per_s": value * w.n_hosts, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32",
+        "data": "synthetic",
+        "config": {"workload": w.name, "n_snapshots": w.n_snapshots, "n_hosts": w.n_hosts,
+                   "batch": w.batch, "sample_requests_per_step": dec},
+        "cpu_baseline": {"value": value, "unit": "decisions/s", "cores": 1, "kind": "oracle",
+                         "sample": f"first {sample} requests of each snapshot against all "
+                                   f"{w.n_hosts} hosts, per step"},
+        "e2e": {"value": value, "unit": "decisions/s", "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    from paper_2503_20591_b200 import binding as nb, build as lib_build, workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    else:
+        dist = None
+        torch.cuda.set_device(0)
+    dev = torch.device("cuda", torch.cuda.current_device())
+    if rank == 0:
+        lib_build.build()
+    if dist is not None:
+        dist.barrier()
+    nb.load_library()
+
+    # ---- inputs: one cluster snapshot per rank, several request batches rotated so that their
+    # total exceeds the L2 cache (weak scaling: every rank places its own full batch) ----
+    w = W.make_config(args.workload, batch=args.batch, n_snapshots=args.snapshots)
+    per_batch_bytes = w.decisions * (16 + 12 + 4)
+    n_rot = max(2, min(12, -(-int(1.3 * L2_BYTES) // per_batch_bytes)))
+    batches = [w.requests] if rank == 0 else []
+    batches += W.extra_request_batches(args.workload, n_rot - len(batches), batch=w.batch,
+                                       n_snapshots=w.n_snapshots, seed0=10_000 + 1000 * rank)
+    d_state = [torch.from_numpy(getattr(w, k)).to(dev).reshape(-1) for k in w.HOST_FIELDS]
+    lim_num, lim_den = torch.from_numpy(w.limit_num), torch.from_numpy(w.limit_den)
+    d_req = [torch.from_numpy(b).to(dev) for b in batches]
+    d_out = [torch.empty((w.n_snapshots, w.batch, 3), dtype=torch.int32, device=dev) for _ in batches]
+    d_found = [torch.empty((w.n_snapshots, w.batch), dtype=torch.int32, device=dev) for _ in batches]
+    workspace = torch.empty(nb.nbos_snapshot_workspace_bytes(w.n_snapshots, w.n_hosts),
+                            dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(i, ev=None):
+        snap = nb.nbos_snapshot_create(w.n_snapshots, w.n_hosts, lim_num, lim_den, *d_state,
+                                       replicas_R=w.replicas_R, workspace=workspace, stream=stream)
+        k = i % n_rot
+        if ev is not None:
+            ev[0].record(stream)
+        nb.nbos_place_batch(snap, d_req[k], d_out[k], d_found[k], stream=stream)
+        if ev is not None:
+            ev[1].record(stream)
+        return snap
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    sampler = ClockSampler(dev.index)
+    snaps = []
+    for i in range(max(3, args.warmup)):
+        snaps.append(step(i))
+    sync_all()
+    for s in snaps:
+        nb.nbos_snapshot_destroy(s)
+    snaps = []
+    kern_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    e0.record(stream)
+    for i in range(args.steps):
+        snaps.append(step(i, kern_events[i]))
+    e1.record(stream)
+    sync_all()
+    sampler.stop()
+    status = nb.nbos_snapshot_status(snaps[-1], stream)
+    for s in snaps:
+        nb.nbos_snapshot_destroy(s)
+    if status != nb.NBOS_OK:
+        raise RuntimeError("device status: " + nb.nbos_strerror(status))
+    ms_total = e0.elapsed_time(e1)
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    kern_ms = statistics.mean(a.elapsed_time(b) for a, b in kern_events)
+    decisions_all = w.decisions * world
+    value = decisions_all / (ms_per_step * 1e-3)
+    clocks = sampler.summary()
+
+    # ---- end to end: host buffers in, host buffers out, through the *_host entry points ----
+    e2e = None
+    if not args.no_e2e:
+        h_state = [torch.from_numpy(getattr(w, k)).reshape(-1) for k in w.HOST_FIELDS]
+        h_req = [torch.from_numpy(b).pin_memory() for b in batches[:2]]
+        h_out = torch.empty((w.n_snapshots, w.batch, 3), dtype=torch.int32).pin_memory()
+        h_found = torch.empty((w.n_snapshots, w.batch), dtype=torch.int32).pin_memory()
+
+        def e2e_step(i):
+            snap = nb.nbos_snapshot_create_host(w.n_snapshots, w.n_hosts, lim_num, lim_den,
+                                                *h_state, replicas_R=w.replicas_R, stream=stream)
+            nb.nbos_place_batch_host(snap, h_req[i % 2], h_out, h_found, stream=stream)
+            nb.nbos_snapshot_destroy(snap)
+
+        e2e_steps = max(3, min(args.steps, 20))
+        for i in range(3):
+            e2e_step(i)
+        sync_all()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for i in range(e2e_steps):
+            e2e_step(i)
+        b.record(stream)
+        sync_all()
+        t = torch.tensor([a.elapsed_time(b)], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item()) / e2e_steps
+        h2d = w.decisions * 16 + 6 * 4 * w.n_snapshots * w.n_hosts + 8 * w.n_snapshots
+        d2h = w.decisions * (12 + 4)
+        e2e = {"value": decisions_all / (e2e_ms * 1e-3), "unit": "decisions/s",
+               "ms_per_step": e2e_ms, "steps": e2e_steps, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "host_memory": "pinned"}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    # ---- integer issue-rate probe, same process, same clocks ----
+    probe = {}
+    for name, mix in (("alu", nb.NBOS_PROBE_MIX_ALU), ("imad", nb.NBOS_PROBE_MIX_IMAD),
+                      ("both", nb.NBOS_PROBE_MIX_BOTH)):
+        nb.nbos_probe_int32_issue(mix, 2048, SM_COUNT_B200 * 8, 256)
+        ops, ms = nb.nbos_probe_int32_issue(mix, 8192, SM_COUNT_B200 * 8, 256)
+        probe[name + "_gops"] = ops / ms / 1e6
+
+    sm_mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    peak_gops = sms * INT32_LANES_PER_SM * sm_mhz * 1e6 / 1e9
+    achieved_gops = ALGORITHMIC_OPS_PER_PAIR * w.pairs / (kern_ms * 1e-3) / 1e9
+    roofline = {
+        "bound": "alu", "kernel": "place_kernel", "achieved": achieved_gops, "peak": peak_gops,
+        "unit": "Gop/s (thread-level INT32 instructions)", "frac": achieved_gops / peak_gops,
+        "peak_source": f"{sms} SMs x {INT32_LANES_PER_SM} INT32 lanes x {sm_mhz:.0f} MHz sampled "
+                       "during the timed region; probe_alu_gops is the same peak measured",
+        "ops_per_pair": ALGORITHMIC_OPS_PER_PAIR, "kernel_ms": kern_ms,
+        "pairs_per_s_kernel": w.pairs / (kern_ms * 1e-3),
+        "traffic": PLACE_KERNEL_DRAM_BYTES_PER_LAUNCH,
+        "stream_gbs": w.decisions * (16 + 12 + 4) / (kern_ms * 1e-3) / 1e9,
+        "probe_alu_gops": probe["alu_gops"], "probe_imad_gops": probe["imad_gops"],
+        "probe_both_gops": probe["both_gops"],
+    }
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        sample = args.cpu_sample or max(16, min(w.batch, (1 << 28) // (w.n_snapshots * w.n_hosts)))
+        dec, dt, res = time_checker(w, sample, 1, 0)
+        same = bool(np.array_equal(res[0], d_out[0][:, :sample].cpu().numpy())
+                    and np.array_equal(res[1], d_found[0][:, :sample].cpu().numpy()))
+        cpu_baseline = {"value": dec / dt, "unit": "decisions/s", "pairs_per_s": dec * w.n_hosts / dt,
+                        "cores": 1, "host_cores_available": os.cpu_count(), "kind": "oracle",
+                        "seconds": dt,
+                        "sample": f"first {sample} requests of each snapshot against all "
+                                  f"{w.n_hosts} hosts, once",
+                        "gpu_output_identical_on_sample": same}
+
+    rot_mib = n_rot * per_batch_bytes / 2**20
+    launches_per_step = 4  # init_stats, scan, emit (derivation) + placement kernel
+    line = {
+        "metric": "placement decisions/sec", "value": value, "unit": "decisions/s",
+        "pairs_per_s": value * w.n_hosts, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+        "config": {"workload": w.name, "n_snapshots": w.n_snapshots, "n_hosts": w.n_hosts,
+                   "batch": w.batch, "pairs_per_step_per_gpu": w.pairs, "replicas_R": w.replicas_R,
+                   "step": "snapshot derivation + placement of one batch",
+                   "l2": f"inputs rotate over {n_rot} request/result batch sets, {rot_mib:.0f} MiB "
+                         f"in total ({'larger' if rot_mib > 126 else 'SMALLER'} than the 126 MiB L2)",
+                   "inputs_sha256": w.sha256()},
+        "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
+        "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -247,3 +247,20 @@ def make_config(index: int, batch: int | None = None, n_snapshots: int | None = 
         off = 0 if seed is None else seed
         return what_if_sweep(n, h, b, "cfg4_what_if_sweep", 1000 + off, 2000 + off)
     raise ValueError(f"no such workload: {index}")
+
+
+def extra_request_batches(index: int, count: int, batch: int | None = None,
+                          n_snapshots: int | None = None, seed0: int = 10_000) -> list:
+    """`count` further request batches [N, B, 4] for benchmark workload `index`, drawn from that
+    workload's request distribution with seeds of their own (seed0 + 100 * index + k). Used to
+    rotate inputs so that successive timed steps do not find their requests in the L2 cache."""
+    n, _, b = CONFIG_SHAPES[index]
+    b = b if batch is None else batch
+    n = n if n_snapshots is None else n_snapshots
+    probs = GPU_ASK_PROBS_SKEWED if index == 2 else GPU_ASK_PROBS_DEFAULT
+    out = []
+    for k in range(count):
+        rng = np.random.Generator(np.random.PCG64(seed0 + 100 * index + k))
+        out.append(np.ascontiguousarray(
+            np.stack([_requests(rng, b, probs) for _ in range(n)]).astype(np.int32)))
+    return out
