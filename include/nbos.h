@@ -190,6 +190,43 @@ int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_hos
                           int64_t batch_per_snapshot, int32_t *out_hosts_host,
                           int32_t *out_found_host, void *cuda_stream);
 
+/*
+ * Placement for callers that are not allowed to allocate device memory. (The paper has no
+ * counterpart; this is a deployment variant of nbos_place_batch with the host-split launch
+ * shape.)
+ *
+ * Who needs it: a scheduler that shares its GPU with a training or serving job which has
+ * already handed all free device memory to its own pool, so that a cudaMalloc here can fail or
+ * evict; and control loops with a latency budget, where the device-wide synchronisation and
+ * the driver lock an allocation may take are not acceptable. nbos_place_batch allocates a
+ * temporary candidate buffer whenever it cuts the hosts into slices (small batches against many
+ * hosts). This entry point computes the same result with that buffer placed in a fixed array
+ * of NBOS_NOALLOC_SCRATCH_BYTES that is part of the library image: every GPU on which the
+ * library is loaded holds those bytes until the process exits. It calls no cudaMalloc,
+ * cudaFree or other allocating routine. Inputs and outputs are still the caller's.
+ *
+ *   host_split   K, number of host slices (1..NBOS_NOALLOC_MAX_SPLIT; 0 = 4). It is lowered to
+ *                what the host count allows. K = 1 uses no candidate buffer at all.
+ *   limit        K * N * batch_per_snapshot * 3 keys (4 bytes each, 8 when the snapshot uses
+ *                64-bit keys) must fit NBOS_NOALLOC_SCRATCH_BYTES; otherwise the call returns
+ *                NBOS_ERR_NO_MEMORY, says so in nbos_last_error_detail(), and launches nothing.
+ *   first call   The first call on each device looks up the array's device address
+ *                (cudaGetSymbolAddress, with that device current). Make that first call during
+ *                start-up, before any stream capture begins.
+ *   sharing      All calls in the process, on all streams, use the same array, and it keeps
+ *                whatever the previous call left. Nothing in it needs clearing: each call writes
+ *                every slot it later reads. But two calls that overlap on the GPU (different
+ *                streams, no dependency between them) race on it and give wrong results: order
+ *                them on one stream or with events.
+ * Other arguments, output and asynchrony as for nbos_place_batch; the snapshot must belong to
+ * the current device.
+ */
+#define NBOS_NOALLOC_SCRATCH_BYTES (8u << 20)
+#define NBOS_NOALLOC_MAX_SPLIT 64
+int nbos_place_batch_noalloc(const nbos_snapshot *snap, const int32_t *requests,
+                             int64_t batch_per_snapshot, int32_t *out_hosts, int32_t *out_found,
+                             void *cuda_stream, int32_t host_split);
+
 /* Synchronises `cuda_stream` and returns the sticky device status of this snapshot: NBOS_OK, or
  * NBOS_ERR_DEVICE_TIMEOUT if some kernel gave up on a bounded wait (its outputs are then
  * undefined). */

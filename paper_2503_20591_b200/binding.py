@@ -36,7 +36,7 @@ NBOS_PROBE_MIX_BOTH = 2
 EXPORTED_SYMBOLS = (
     "nbos_snapshot_workspace_bytes", "nbos_snapshot_create", "nbos_snapshot_create_host",
     "nbos_snapshot_destroy", "nbos_snapshot_get_info", "nbos_place_batch", "nbos_place_batch_ex",
-    "nbos_place_batch_host", "nbos_snapshot_status", "nbos_strerror", "nbos_last_error_detail",
+    "nbos_place_batch_host", "nbos_place_batch_noalloc", "nbos_snapshot_status", "nbos_strerror", "nbos_last_error_detail",
     "nbos_probe_int32_issue", "nbos_probe_wait_timeout",
 )
 
@@ -102,6 +102,7 @@ def load_library() -> ctypes.CDLL:
     lib.nbos_place_batch.argtypes = [vp, vp, i64, vp, vp, vp]
     lib.nbos_place_batch_ex.argtypes = [vp, vp, i64, vp, vp, vp, P(nbos_launch_config)]
     lib.nbos_place_batch_host.argtypes = [vp, vp, i64, vp, vp, vp]
+    lib.nbos_place_batch_noalloc.argtypes = [vp, vp, i64, vp, vp, vp, ctypes.c_int32]
     lib.nbos_snapshot_status.argtypes = [vp, vp]
     lib.nbos_strerror.argtypes = [ctypes.c_int]
     lib.nbos_strerror.restype = ctypes.c_char_p
@@ -286,6 +287,27 @@ def nbos_place_batch_host(snap: Snapshot, requests, out_hosts, out_found=None, s
         raise ValueError("out_found must hold n_snapshots * batch values")
     _check(lib.nbos_place_batch_host(snap.handle, _ptr(requests), b, _ptr(out_hosts),
                                      _ptr(out_found), _stream_ptr(stream)))
+
+
+def nbos_place_batch_noalloc(snap: Snapshot, requests, out_hosts, out_found=None, stream=None,
+                             host_split: int = 0) -> None:
+    """Same result as nbos_place_batch, for callers that must not allocate device memory (their
+    GPU memory belongs to another pool, or an allocation's synchronisation does not fit their
+    latency budget): the slice candidates live in a fixed array inside the library. This wrapper
+    allocates nothing either; it only passes pointers. Calls that overlap on the GPU race on the
+    shared array; batches beyond the array's size raise NbosError (NBOS_ERR_NO_MEMORY)."""
+    lib = load_library()
+    _i32(requests, "requests", "cuda")
+    _i32(out_hosts, "out_hosts", "cuda")
+    if out_found is not None:
+        _i32(out_found, "out_found", "cuda")
+    b = _batch_of(snap, requests)
+    if out_hosts.numel() != snap.n_snapshots * b * 3:
+        raise ValueError("out_hosts must hold n_snapshots * batch * 3 values")
+    if out_found is not None and out_found.numel() != snap.n_snapshots * b:
+        raise ValueError("out_found must hold n_snapshots * batch values")
+    _check(lib.nbos_place_batch_noalloc(snap.handle, _ptr(requests), b, _ptr(out_hosts),
+                                        _ptr(out_found), _stream_ptr(stream), host_split))
 
 
 def nbos_probe_int32_issue(mix: int, iters: int, blocks: int, threads: int, stream=None):

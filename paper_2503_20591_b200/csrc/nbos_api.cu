@@ -288,6 +288,23 @@ int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_hos
     return NBOS_OK;
 }
 
+int nbos_place_batch_noalloc(const nbos_snapshot *snap, const int32_t *requests,
+                             int64_t batch_per_snapshot, int32_t *out_hosts, int32_t *out_found,
+                             void *cuda_stream, int32_t host_split)
+{
+    if (!snap) return fail(NBOS_ERR_INVALID_ARG, "snapshot is NULL");
+    if (batch_per_snapshot < 0 || batch_per_snapshot > ((int64_t)1 << 40) / snap->N)
+        return fail(NBOS_ERR_INVALID_ARG, "batch_per_snapshot out of range");
+    if (host_split < 0 || host_split > NBOS_NOALLOC_MAX_SPLIT)
+        return fail(NBOS_ERR_INVALID_ARG, "host_split must be 0 (default) or 1..%d", NBOS_NOALLOC_MAX_SPLIT);
+    if (batch_per_snapshot == 0) return NBOS_OK;
+    if (!requests || !out_hosts) return fail(NBOS_ERR_INVALID_ARG, "requests / out_hosts is NULL");
+    if (!aligned(requests, 16)) return fail(NBOS_ERR_INVALID_ARG, "requests is not 16-byte aligned");
+    if (!aligned(out_hosts, 4) || !aligned(out_found, 4)) return fail(NBOS_ERR_INVALID_ARG, "output not 4-byte aligned");
+    return launch_place_static(snap, requests, batch_per_snapshot, out_hosts, out_found,
+                               static_cast<cudaStream_t>(cuda_stream), host_split);
+}
+
 int nbos_snapshot_status(const nbos_snapshot *snap, void *cuda_stream)
 {
     if (!snap) return fail(NBOS_ERR_INVALID_ARG, "snapshot is NULL");

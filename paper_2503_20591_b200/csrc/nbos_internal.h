@@ -72,5 +72,10 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
                  int32_t *d_out_hosts, int32_t *d_out_found, cudaStream_t stream,
                  const nbos_launch_config *cfg);
 
+// Host-split placement whose candidate buffer is a fixed array inside the module (no allocation).
+int launch_place_static(const nbos_snapshot *s, const int32_t *d_requests, int64_t batch,
+                        int32_t *d_out_hosts, int32_t *d_out_found, cudaStream_t stream,
+                        int host_split);
+
 }  // namespace nbos
 #endif

@@ -22,6 +22,8 @@
 // sticky status word and leaves without touching the barrier again.
 #include <limits.h>
 
+#include <mutex>
+
 #include "nbos_internal.h"
 
 namespace nbos {
@@ -515,6 +517,123 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
     }
     if (p.cand) cudaFreeAsync(p.cand, stream);
     if (e != cudaSuccess) return cuda_fail(e, "placement launch");
+    return NBOS_OK;
+}
+
+
+// ---- placement without any allocation ------------------------------------------------------
+// The host-split launch shape needs a candidate buffer (K slices x requests x 3 keys). The
+// ordinary entry points take it from the stream-ordered allocator; this variant keeps it in a
+// fixed array that is part of the loaded module, for callers that must not allocate.
+namespace {
+
+constexpr size_t kStaticCandBytes = NBOS_NOALLOC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_cand[kStaticCandBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void *g_static_cand_ptr[kMaxDevices] = {};  // device address of g_static_cand, per device
+
+// Host code cannot use the name g_static_cand as a pointer: on the host it only stands for the
+// symbol. The device address is looked up once per device, with that device current.
+int static_cand_address(int device, void **out)
+{
+    if (device < 0 || device >= kMaxDevices) return fail(NBOS_ERR_INVALID_ARG, "device index %d not supported", device);
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_cand_ptr[device]) {
+        void *ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_cand);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(static candidate buffer)");
+        if (!ptr) return fail(NBOS_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
+        g_static_cand_ptr[device] = ptr;
+    }
+    *out = g_static_cand_ptr[device];
+    return NBOS_OK;
+}
+
+}  // namespace
+
+int launch_place_static(const nbos_snapshot *s, const int32_t *d_requests, int64_t batch,
+                        int32_t *d_out_hosts, int32_t *d_out_found, cudaStream_t stream,
+                        int host_split)
+{
+    const long long total = (long long)s->N * batch;
+    if (total == 0) return NBOS_OK;
+    int device = -1;
+    NBOS_CUDA_TRY(cudaGetDevice(&device));
+    if (device != s->device)
+        return fail(NBOS_ERR_INVALID_ARG, "snapshot was created on device %d, current device is %d", s->device, device);
+    const bool k64 = s->key.key_bits == 64;
+    const int key_bytes = k64 ? 8 : 4;
+    const int pair_bytes = k64 ? 16 : 8;
+
+    // host slices: K tiles-aligned slices of the padded host table
+    int K = host_split ? host_split : 4;
+    if (K > s->Hpad / 32) K = s->Hpad / 32;
+    if (K < 1) K = 1;
+    int T = (s->Hpad / K) / 32 * 32;
+    if (T > 1024) T = 1024;
+    if (T < 32) T = 32;
+    const int tiles_total = (s->Hpad + T - 1) / T;
+    if (K > tiles_total) K = tiles_total;
+
+    const size_t cand_bytes = (size_t)K * (size_t)total * 3 * key_bytes;
+    if (K > 1 && cand_bytes > kStaticCandBytes)
+        return fail(NBOS_ERR_NO_MEMORY,
+                    "nbos_place_batch_noalloc: %lld requests x %d host slices need %zu bytes of candidates, "
+                    "the built-in buffer holds %zu; use fewer slices, a smaller batch, or nbos_place_batch",
+                    total, K, cand_bytes, kStaticCandBytes);
+    void *cand = nullptr;
+    int rc = static_cand_address(device, &cand);
+    if (rc) return rc;
+
+    const int L = 32;  // small batches are what this shape is for: one warp per request group
+    KernelFn fn = k64 ? pick_kernel<unsigned long long, 4>(L) : pick_kernel<unsigned int, 8>(L);
+    const size_t smem = (size_t)kStages * T * (16 + pair_bytes) + 2 * kStages * 8 + 16;
+    NBOS_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int per_sm = 0;
+    NBOS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kThreads, smem));
+    if (per_sm < 1) return fail(NBOS_ERR_CUDA, "placement kernel does not fit on an SM");
+    const int groups = kComputeThreads / L;
+    long long req_ctas = (total + groups - 1) / groups;
+    long long cap = (long long)s->sm_count * per_sm / K;
+    if (cap < 1) cap = 1;
+    if (req_ctas > cap) req_ctas = cap;
+
+    PlaceParams p;
+    p.feas = s->d_feas;
+    p.ab = s->d_ab;
+    p.requests = reinterpret_cast<const int4 *>(d_requests);
+    p.out_hosts = d_out_hosts;
+    p.out_found = d_out_found;
+    p.cand = K > 1 ? cand : nullptr;
+    p.status = s->d_status;
+    p.B = batch;
+    p.total = total;
+    p.N = s->N;
+    p.Hpad = s->Hpad;
+    p.tile_hosts = T;
+    p.tiles_total = tiles_total;
+    p.K = K;
+    p.req_ctas = (int)req_ctas;
+    p.id_mask = (1u << s->key.bits_id) - 1u;
+    p.max_q = k64 ? 4 : 8;
+
+    // Nothing in the buffer has to start at zero: the placement kernel writes all K * total * 3
+    // candidate slots of this call before the merge kernel (next on the stream) reads them.
+    fn<<<(unsigned int)(req_ctas * K), kThreads, smem, stream>>>(p);
+    NBOS_CUDA_TRY(cudaGetLastError());
+    if (K > 1) {
+        long long blocks = (total + 255) / 256;
+        if (blocks > (long long)s->sm_count * 8) blocks = (long long)s->sm_count * 8;
+        if (k64)
+            merge_kernel<unsigned long long><<<(unsigned int)blocks, 256, 0, stream>>>(
+                static_cast<const unsigned long long *>(cand), K, total, p.id_mask, d_out_hosts, d_out_found);
+        else
+            merge_kernel<unsigned int><<<(unsigned int)blocks, 256, 0, stream>>>(
+                static_cast<const unsigned int *>(cand), K, total, p.id_mask, d_out_hosts, d_out_found);
+        NBOS_CUDA_TRY(cudaGetLastError());
+    }
     return NBOS_OK;
 }
 
