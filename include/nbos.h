@@ -105,6 +105,11 @@ typedef struct nbos_snapshot_info {
     int32_t key_bits;                    /* 32 or 64: width of the ranking key in use       */
     int32_t bits_idle, bits_sr, bits_id; /* field widths inside the key                     */
     int32_t key_order, flags, replicas_R;
+    int32_t packed_test; /* 0: capacities too wide for the packed test; 1: packed, one guard
+                          * mask; 2: packed, one guard mask per word                        */
+    int32_t static_key;  /* 1: every host has the same key slope, hosts rank the same for all g */
+    int32_t presorted;   /* 1: the host table is stored in ascending key order              */
+    int32_t reserved;
     int64_t workspace_bytes;
 } nbos_snapshot_info;
 
@@ -118,6 +123,10 @@ typedef struct nbos_snapshot_info {
  *                      merge kernel.
  *   tile_hosts         hosts per shared-memory tile (multiple of 32).
  *   grid_blocks        thread blocks along the request dimension (per host slice).
+ *   pair_mode          how a (request, host) pair is evaluated when the snapshot has 32-bit keys:
+ *                      0 = the fastest form the snapshot allows; 1 = four separate capacity
+ *                      compares; 2 = packed capacity test with the key computed per pair (even if
+ *                      the snapshot would allow ranking by the host part of the key alone).
  */
 typedef struct nbos_launch_config {
     int32_t lanes_per_request;
@@ -125,7 +134,8 @@ typedef struct nbos_launch_config {
     int32_t host_split;
     int32_t tile_hosts;
     int32_t grid_blocks;
-    int32_t reserved[3]; /* must be 0 */
+    int32_t pair_mode;
+    int32_t reserved[2]; /* must be 0 */
 } nbos_launch_config;
 
 /* Device bytes nbos_snapshot_create needs in `workspace` for this N and H (Section 3.4.1 state

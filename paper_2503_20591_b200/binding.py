@@ -61,6 +61,8 @@ class nbos_snapshot_info(ctypes.Structure):
         ("hosts_padded", ctypes.c_int32), ("key_bits", ctypes.c_int32),
         ("bits_idle", ctypes.c_int32), ("bits_sr", ctypes.c_int32), ("bits_id", ctypes.c_int32),
         ("key_order", ctypes.c_int32), ("flags", ctypes.c_int32), ("replicas_R", ctypes.c_int32),
+        ("packed_test", ctypes.c_int32), ("static_key", ctypes.c_int32),
+        ("presorted", ctypes.c_int32), ("reserved", ctypes.c_int32),
         ("workspace_bytes", ctypes.c_int64),
     ]
 
@@ -69,7 +71,8 @@ class nbos_launch_config(ctypes.Structure):
     _fields_ = [
         ("lanes_per_request", ctypes.c_int32), ("requests_per_lane", ctypes.c_int32),
         ("host_split", ctypes.c_int32), ("tile_hosts", ctypes.c_int32),
-        ("grid_blocks", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3),
+        ("grid_blocks", ctypes.c_int32), ("pair_mode", ctypes.c_int32),
+        ("reserved", ctypes.c_int32 * 2),
     ]
 
 
@@ -327,10 +330,11 @@ def nbos_probe_wait_timeout(limit_ns: int, stream=None):
 
 
 def launch_config(lanes_per_request=0, requests_per_lane=0, host_split=0, tile_hosts=0,
-                  grid_blocks=0) -> nbos_launch_config:
+                  grid_blocks=0, pair_mode=0) -> nbos_launch_config:
     c = nbos_launch_config()
     c.lanes_per_request, c.requests_per_lane = lanes_per_request, requests_per_lane
     c.host_split, c.tile_hosts, c.grid_blocks = host_split, tile_hosts, grid_blocks
+    c.pair_mode = pair_mode
     return c
 
 

@@ -41,7 +41,9 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
     __shared__ unsigned int s_err;
     __shared__ int s_idle_max, s_g_min;
     __shared__ unsigned long long s_sub_max;
+    __shared__ int s_max4[4];
     const int n = blockIdx.y;
+    if (threadIdx.x < 4) s_max4[threadIdx.x] = threadIdx.x == 0 ? -1 : 0;
     if (threadIdx.x < 16) s_mask[threadIdx.x] = 0ull;
     if (threadIdx.x == 0) {
         s_err = 0u;
@@ -54,6 +56,7 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
     unsigned int err = 0u;
     int idle_max = 0, g_min = INT_MAX;
     unsigned long long sub_max = 0ull;
+    int max_gcap = -1, max_av = 0, max_ac = 0, max_am = 0;
     for (int h = blockIdx.x * blockDim.x + threadIdx.x; h < a.H; h += gridDim.x * blockDim.x) {
         const size_t i = (size_t)n * a.H + h;
         const int G = a.G[i], S = a.S[i], C = a.C[i];
@@ -68,11 +71,19 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
         idle_max = max(idle_max, G - C);
         const int gm = derive_gmax(G, S, C, lim.x, lim.y, a.R, a.flags);
         if (gm >= 0) sub_max = max(sub_max, (unsigned long long)S + (unsigned long long)gm);
+        max_gcap = max(max_gcap, gm);
+        max_av = max(max_av, a.AV[i]);
+        max_ac = max(max_ac, a.AC[i]);
+        max_am = max(max_am, a.AM[i]);
     }
     if (err) atomicOr(&s_err, err);
     atomicMax(&s_idle_max, idle_max);
     atomicMin(&s_g_min, g_min);
     atomicMax(&s_sub_max, sub_max);
+    atomicMax(&s_max4[0], max_gcap);
+    atomicMax(&s_max4[1], max_av);
+    atomicMax(&s_max4[2], max_ac);
+    atomicMax(&s_max4[3], max_am);
     __syncthreads();
     SnapStats *st = a.stats + n;
     if (threadIdx.x < 16 && s_mask[threadIdx.x]) atomicOr(&st->g_mask[threadIdx.x], s_mask[threadIdx.x]);
@@ -81,6 +92,10 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
         atomicMax(&st->idle_max, s_idle_max);
         atomicMin(&st->g_min, s_g_min);
         atomicMax(&st->sub_max, s_sub_max);
+        atomicMax(&st->max_gcap, s_max4[0]);
+        atomicMax(&st->max_av, s_max4[1]);
+        atomicMax(&st->max_ac, s_max4[2]);
+        atomicMax(&st->max_am, s_max4[3]);
     }
 }
 
@@ -90,6 +105,7 @@ __global__ void init_stats_kernel(SnapStats *stats, int n)
     if (i < n) {
         SnapStats z = {};
         z.g_min = INT_MAX;
+        z.max_gcap = -1;
         stats[i] = z;
     }
 }
@@ -98,12 +114,16 @@ struct EmitArgs {
     const int32_t *G, *S, *C, *AV, *AC, *AM;
     const int2 *limits;
     const long long *lambda;  // per snapshot
-    int4 *feas;
+    int4 *feas;                 // records in host-index order (staging)
     void *ab;
+    unsigned long long *sortkey;  // [N][Hpad] visiting-order key: A, or near-max for hosts that take nothing
     int H, Hpad, R, flags, key_order;
     int idle_max;             // over all snapshots: the idle field stores idle_max - (G - C)
     int bits_idle, bits_sr, bits_id;
 };
+
+constexpr int kSortMaxHosts = 8192;  // largest (padded, power of two) table sorted in shared memory
+constexpr unsigned long long kSortNever = 0xFFFFFFFFFFFFFFFEull;  // hosts that take nothing go last
 
 // grid (ceil(Hpad / 256), N). One record per (padded) host.
 template <typename KeyT, typename PairT>
@@ -114,6 +134,7 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
     if (h >= a.Hpad) return;
     int4 f = make_int4(-1, 0, 0, 0);  // padding host: takes nothing
     KeyT A = (KeyT)h, B = 0;
+    unsigned long long sk = kSortNever;
     if (h < a.H) {
         const size_t i = (size_t)n * a.H + h;
         const int G = a.G[i], S = a.S[i], C = a.C[i];
@@ -131,13 +152,91 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
                 A = (idle_inv << (a.bits_sr + a.bits_id)) + (sr0 << a.bits_id) + (KeyT)h;
                 B = w << a.bits_id;
             }
+            sk = (unsigned long long)A;
         }
     }
+    a.sortkey[(size_t)n * a.Hpad + h] = sk;
     a.feas[(size_t)n * a.Hpad + h] = f;
     PairT p;
     p.x = A;
     p.y = B;
     reinterpret_cast<PairT *>(a.ab)[(size_t)n * a.Hpad + h] = p;
+}
+
+// Visiting order. One block per snapshot sorts (sortkey, position) in shared memory (bitonic,
+// n2 = power of two >= Hpad) and writes the permutation. Hosts are visited in ascending order of
+// their key at g = 0, which makes later hosts rarely displace an earlier best-three entry.
+__global__ void __launch_bounds__(1024) sort_kernel(const unsigned long long *sortkey, unsigned int *perm,
+                                                    int Hpad, int n2)
+{
+    extern __shared__ __align__(16) unsigned char sort_smem[];
+    unsigned long long *keys = reinterpret_cast<unsigned long long *>(sort_smem);
+    unsigned int *pos = reinterpret_cast<unsigned int *>(sort_smem + (size_t)n2 * 8);
+    const size_t base = (size_t)blockIdx.x * Hpad;
+    for (int i = threadIdx.x; i < n2; i += blockDim.x) {
+        keys[i] = i < Hpad ? sortkey[base + i] : 0xFFFFFFFFFFFFFFFFull;
+        pos[i] = (unsigned int)i;
+    }
+    __syncthreads();
+    for (int k = 2; k <= n2; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = threadIdx.x; i < n2; i += blockDim.x) {
+                const int other = i ^ j;
+                if (other > i) {
+                    const bool up = (i & k) == 0;
+                    const unsigned long long a = keys[i], b = keys[other];
+                    if ((a > b) == up) {
+                        keys[i] = b;
+                        keys[other] = a;
+                        const unsigned int t = pos[i];
+                        pos[i] = pos[other];
+                        pos[other] = t;
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    for (int i = threadIdx.x; i < Hpad; i += blockDim.x) perm[base + i] = pos[i];
+}
+
+__global__ void identity_perm_kernel(unsigned int *perm, int Hpad, size_t total)
+{
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < total) perm[i] = (unsigned int)(i % Hpad);
+}
+
+struct FinalizeArgs {
+    const int4 *tmp_feas;
+    const void *tmp_ab;
+    const unsigned int *perm;
+    int4 *feas;
+    void *ab;
+    uint4 *pk;
+    int Hpad;
+    PackLayout pack;
+};
+
+// grid (ceil(Hpad / 256), N): gather the records into visiting order and build the packed form.
+template <typename PairT>
+__global__ void __launch_bounds__(256) finalize_kernel(const FinalizeArgs a)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= a.Hpad) return;
+    const size_t base = (size_t)blockIdx.y * a.Hpad;
+    const unsigned int src = a.perm[base + j];
+    const int4 f = a.tmp_feas[base + src];
+    const PairT p = reinterpret_cast<const PairT *>(a.tmp_ab)[base + src];
+    a.feas[base + j] = f;
+    reinterpret_cast<PairT *>(a.ab)[base + j] = p;
+    if (a.pack.enabled) {
+        const unsigned int cap[4] = {(unsigned int)(f.x + 1), (unsigned int)f.y, (unsigned int)f.z,
+                                     (unsigned int)f.w};
+        unsigned int w[2] = {a.pack.guards, a.pack.guards1};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) w[a.pack.fword[c]] |= cap[c] << a.pack.fshift[c];
+        a.pk[base + j] = make_uint4(w[0], w[1], (unsigned int)p.x, (unsigned int)p.y);
+    }
 }
 
 int bits_for(unsigned long long max_value)
@@ -173,6 +272,11 @@ Layout workspace_layout(int N, int Hpad)
     l.off_stats = o;   o = up(o + (size_t)N * sizeof(SnapStats));
     l.off_feas = o;    o = up(o + (size_t)N * Hpad * sizeof(int4));
     l.off_ab = o;      o = up(o + (size_t)N * Hpad * sizeof(ulonglong2));
+    l.off_pk = o;      o = up(o + (size_t)N * Hpad * sizeof(uint4));
+    l.off_tmp_feas = o; o = up(o + (size_t)N * Hpad * sizeof(int4));
+    l.off_tmp_ab = o;  o = up(o + (size_t)N * Hpad * sizeof(ulonglong2));
+    l.off_sortkey = o; o = up(o + (size_t)N * Hpad * sizeof(unsigned long long));
+    l.off_perm = o;    o = up(o + (size_t)N * Hpad * sizeof(unsigned int));
     l.total = o;
     return l;
 }
@@ -247,12 +351,54 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     const int total_bits = k.bits_idle + k.bits_sr + k.bits_id;
     if (total_bits > 63) return fail(NBOS_ERR_RANGE, "ranking key needs %d bits (max 63)", total_bits);
     k.key_bits = (total_bits <= 31 && !(s->flags & NBOS_FORCE_KEY64)) ? 32 : 64;
+    k.static_key = 1;
+    int fmax[4] = {0, 0, 0, 0};
+    for (int n = 0; n < N; ++n) {
+        const SnapStats &st = h_stats[n];
+        int distinct_g = 0;
+        for (int w = 0; w < 16; ++w) distinct_g += __builtin_popcountll(st.g_mask[w]);
+        if (distinct_g > 1) k.static_key = 0;
+        if (st.max_gcap > fmax[0]) fmax[0] = st.max_gcap;
+        if (st.max_av > fmax[1]) fmax[1] = st.max_av;
+        if (st.max_ac > fmax[2]) fmax[2] = st.max_ac;
+        if (st.max_am > fmax[3]) fmax[3] = st.max_am;
+    }
     s->key = k;
+
+    // packed capacity test: the two widest components become the high fields of the two words
+    PackLayout pk = {};
+    if (k.key_bits == 32) {
+        int width[4], order[4] = {0, 1, 2, 3};
+        width[0] = bits_for((unsigned long long)fmax[0] + 2);  // stored +1, and one more for "fits nowhere"
+        for (int c = 1; c < 4; ++c) width[c] = fmax[c] ? bits_for((unsigned long long)fmax[c]) : 1;
+        for (int i = 0; i < 4; ++i)
+            for (int j = i + 1; j < 4; ++j)
+                if (width[order[j]] > width[order[i]]) { int t = order[i]; order[i] = order[j]; order[j] = t; }
+        // widest with narrowest in word 0, the middle two in word 1
+        const int hi0 = width[order[0]], lo0 = width[order[3]], hi1 = width[order[1]], lo1 = width[order[2]];
+        int lo_a = -1, lo_b = -1;
+        if (hi0 + lo1 + 2 <= 32) lo_a = lo_b = lo1;                              // same guard positions in both words
+        else if (hi0 + lo0 + 2 <= 32 && hi1 + lo1 + 2 <= 32) { lo_a = lo0; lo_b = lo1; }  // each word its own
+        if (lo_a >= 0) {
+            pk.enabled = 1;
+            pk.guards = 0x80000000u | (1u << lo_a);
+            pk.guards1 = 0x80000000u | (1u << lo_b);
+            for (int c = 0; c < 4; ++c) pk.fmax[c] = fmax[c];
+            pk.fword[order[0]] = 0; pk.fshift[order[0]] = lo_a + 1;
+            pk.fword[order[3]] = 0; pk.fshift[order[3]] = 0;
+            pk.fword[order[1]] = 1; pk.fshift[order[1]] = lo_b + 1;
+            pk.fword[order[2]] = 1; pk.fshift[order[2]] = 0;
+        }
+    }
+    s->pack = pk;
 
     NBOS_CUDA_TRY(cudaMemcpyAsync(d_lambda, h_lambda, sizeof(long long) * (size_t)N,
                                   cudaMemcpyHostToDevice, stream));
-    EmitArgs ea{d_G, d_S, d_C, d_AV, d_AC, d_AM, d_limits, d_lambda,
-                reinterpret_cast<int4 *>(ws + lay.off_feas), ws + lay.off_ab,
+    int4 *tmp_feas = reinterpret_cast<int4 *>(ws + lay.off_tmp_feas);
+    void *tmp_ab = ws + lay.off_tmp_ab;
+    unsigned long long *sortkey = reinterpret_cast<unsigned long long *>(ws + lay.off_sortkey);
+    unsigned int *perm = reinterpret_cast<unsigned int *>(ws + lay.off_perm);
+    EmitArgs ea{d_G, d_S, d_C, d_AV, d_AC, d_AM, d_limits, d_lambda, tmp_feas, tmp_ab, sortkey,
                 H, Hpad, s->R, s->flags, s->key_order, idle_max, k.bits_idle, k.bits_sr, k.bits_id};
     dim3 grid((Hpad + 255) / 256, N);
     if (k.key_bits == 32)
@@ -260,9 +406,32 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     else
         emit_kernel<unsigned long long, ulonglong2><<<grid, 256, 0, stream>>>(ea);
     NBOS_CUDA_TRY(cudaGetLastError());
+
+    // visiting order
+    int n2 = 32;
+    while (n2 < Hpad) n2 <<= 1;
+    s->presorted = n2 <= kSortMaxHosts;
+    if (s->presorted) {
+        const size_t sort_smem = (size_t)n2 * 12;
+        NBOS_CUDA_TRY(cudaFuncSetAttribute(sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sort_smem));
+        const int sort_threads = n2 / 2 > 1024 ? 1024 : n2 / 2 < 32 ? 32 : n2 / 2;
+        sort_kernel<<<N, sort_threads, sort_smem, stream>>>(sortkey, perm, Hpad, n2);
+    } else {
+        const size_t total = (size_t)N * Hpad;
+        identity_perm_kernel<<<(unsigned int)((total + 255) / 256), 256, 0, stream>>>(perm, Hpad, total);
+    }
+    NBOS_CUDA_TRY(cudaGetLastError());
+    FinalizeArgs fa{tmp_feas, tmp_ab, perm, reinterpret_cast<int4 *>(ws + lay.off_feas), ws + lay.off_ab,
+                    reinterpret_cast<uint4 *>(ws + lay.off_pk), Hpad, pk};
+    if (k.key_bits == 32)
+        finalize_kernel<uint2><<<grid, 256, 0, stream>>>(fa);
+    else
+        finalize_kernel<ulonglong2><<<grid, 256, 0, stream>>>(fa);
+    NBOS_CUDA_TRY(cudaGetLastError());
     s->d_status = reinterpret_cast<unsigned int *>(ws + lay.off_status);
     s->d_feas = reinterpret_cast<const int4 *>(ws + lay.off_feas);
     s->d_ab = ws + lay.off_ab;
+    s->d_pk = reinterpret_cast<const uint4 *>(ws + lay.off_pk);
     return NBOS_OK;
 }
 

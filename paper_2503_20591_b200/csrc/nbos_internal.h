@@ -27,6 +27,7 @@ struct SnapStats {                 // one per snapshot, filled by the scan kerne
     int g_min;                     // min over hosts with G >= 1 of G (INT_MAX if none)
     int pad;
     unsigned long long sub_max;    // max over hosts that can take something of S + gmax
+    int max_gcap, max_av, max_ac, max_am;  // maxima of gmax and of the three capacities
     unsigned long long g_mask[16]; // bit G set if some host has G GPUs (G in 1..1023)
 };
 enum : unsigned int {
@@ -36,7 +37,8 @@ enum : unsigned int {
 };
 
 struct Layout {
-    size_t off_status, off_limits, off_lambda, off_stats, off_feas, off_ab, total;
+    size_t off_status, off_limits, off_lambda, off_stats, off_feas, off_ab, off_pk;
+    size_t off_tmp_feas, off_tmp_ab, off_sortkey, off_perm, total;
 };
 Layout workspace_layout(int n_snapshots, int hosts_padded);
 inline int pad_hosts(int h) { return (h + 31) & ~31; }
@@ -44,6 +46,21 @@ inline int pad_hosts(int h) { return (h + 31) & ~31; }
 struct KeyLayout {
     int key_bits;  // 32 or 64
     int bits_idle, bits_sr, bits_id;
+    int static_key;  // 1 if B is the same for every host that can take a request: order = order of A
+};
+
+// Two-compares-per-subtraction encoding of the four capacity tests. Components: 0 = GPUs
+// (stored as gmax + 1 against ask + 1, so that 0 means "takes nothing"), 1 = VRAM, 2 = millicpus,
+// 3 = memory. Each 32-bit word holds a low field [0, lo_bits) with its guard bit at lo_bits and
+// a high field from lo_bits + 1 with its guard bit at 31. host_word - request_word keeps a
+// guard bit set exactly when capacity >= ask in that field.
+struct PackLayout {
+    int enabled;
+    int fmax[4];    // largest ask that any host could satisfy, per component
+    int fword[4];   // which word (0 / 1) holds the component
+    int fshift[4];  // bit position of the component inside its word
+    unsigned int guards;    // guard bits of word 0
+    unsigned int guards1;   // guard bits of word 1 (equal to `guards` when the layouts coincide)
 };
 
 }  // namespace nbos
@@ -55,8 +72,12 @@ struct nbos_snapshot {
     size_t workspace_bytes;
     bool owns_workspace;
     unsigned int *d_status;
+    // tables in visiting order (hosts sorted by ascending A when the table is small enough)
     const int4 *d_feas;   // [N][Hpad] (gmax, vram_gb, millicpus, mem_mb)
     const void *d_ab;     // [N][Hpad] uint2 (32-bit keys) or ulonglong2 (64-bit keys): (A, B)
+    const uint4 *d_pk;    // [N][Hpad] (word0, word1, A, B), only when pack.enabled
+    nbos::PackLayout pack;
+    int presorted;
     int device, sm_count;
 };
 

@@ -23,21 +23,40 @@
 #include <limits.h>
 
 #include <mutex>
+#include <type_traits>
 
 #include "nbos_internal.h"
 
 namespace nbos {
 namespace {
 
-constexpr int kComputeThreads = 256;
+constexpr int kComputeThreads = 224;
 constexpr int kComputeWarps = kComputeThreads / 32;
-constexpr int kThreads = kComputeThreads + 32;  // + the copy warp
+constexpr int kThreads = kComputeThreads + 32;  // + the copy warp = 256
+
+// How a (request, host) pair is evaluated; chosen per snapshot when it is derived.
+enum : int {
+    MODE_KEY64 = 0,          // 64-bit keys, plain C++ compares                (records: feas + ab)
+    MODE_PLAIN = 1,          // 32-bit keys, four compares + multiply-add       (records: feas + ab)
+    MODE_PACKED = 2,         // 32-bit keys, two packed subtractions + multiply-add   (records: pk)
+    MODE_PACKED_STATIC = 3,  // as 2, but B is the same on every host: rank by A alone (records: pk)
+    MODE_PACKED2 = 4,        // as 2, the two words have their low guard bit at different positions
+    MODE_PACKED2_STATIC = 5, // as 3, likewise
+    MODE_COUNT = 6,
+};
+__host__ __device__ constexpr bool mode_is_packed(int mode) { return mode >= MODE_PACKED; }
+__host__ __device__ constexpr bool mode_is_static(int mode) { return mode == MODE_PACKED_STATIC || mode == MODE_PACKED2_STATIC; }
+__host__ __device__ constexpr bool mode_two_masks(int mode) { return mode == MODE_PACKED2 || mode == MODE_PACKED2_STATIC; }
+__host__ __device__ constexpr int mode_record_bytes(int mode) { return mode == MODE_KEY64 ? 32 : mode == MODE_PLAIN ? 24 : 16; }
+__host__ __device__ constexpr int mode_max_q(int mode) { return mode == MODE_KEY64 ? 4 : 8; }
 constexpr int kStages = 3;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 struct PlaceParams {
     const int4 *feas;       // [N][Hpad]
     const void *ab;         // [N][Hpad] pairs (A, B)
+    const uint4 *pk;        // [N][Hpad] (word0, word1, A, B), packed modes
+    PackLayout pack;
     const int4 *requests;   // [N * B]
     int32_t *out_hosts;     // [N * B * 3]
     int32_t *out_found;     // [N * B] or null
@@ -143,8 +162,8 @@ __device__ __forceinline__ void insert3(KeyT &t1, KeyT &t2, KeyT &t3, KeyT k)
 
 // ---- the list of passes a block makes over its share of the requests ----------------------
 // A block owns the flattened request range [lo, hi) of [0, N * B). It is cut at snapshot
-// boundaries and then into passes of Q * groups requests, Q the largest power of two <= max_q
-// that still fills every lane (or 1 for the ragged tail). Copy warp and compute threads walk
+// boundaries and then into passes of up to Q * groups requests: full passes of max_q, then one
+// pass with the smallest power of two that covers the rest. Copy warp and compute threads walk
 // the same list.
 struct PassList {
     long long cursor, hi, B;
@@ -156,8 +175,10 @@ struct PassList {
         long long end = (long long)(n + 1) * B;
         if (end > hi) end = hi;
         const long long rem = end - cursor;
+        // the smallest power of two that covers what is left, but at least 2 requests per lane: a
+        // half-empty pass of 2 is cheaper than a full pass of 1 (per-host overhead dominates there)
         q = max_q;
-        while (q > 1 && (long long)q * groups > rem) q >>= 1;
+        while (q > 2 && (long long)(q >> 1) * groups >= rem) q >>= 1;
         const long long cap = (long long)q * groups;
         count = (int)(rem < cap ? rem : cap);
         first = cursor;  // flattened index n * B + r
@@ -177,33 +198,146 @@ __device__ __forceinline__ void block_request_range(const PlaceParams &p, int cr
     if (hi > p.total) hi = p.total;
 }
 
+// ---- the pair step --------------------------------------------------------------------------
+// Fast path of the 32-bit modes: decide whether this pair would enter the request's best three
+// and, if so, bump a per-thread counter (a predicated FADD, off the integer pipe). The update
+// itself is rare and happens once per host behind a single branch (see run_pass). The inline
+// PTX pins the instruction selection: compares chained through one predicate, the subtractions
+// and the key on the multiply pipe.
+__device__ __forceinline__ void pair_plain(float &cnt, unsigned int t3, int g, int v, int c, int m,
+                                           const int4 &f, const uint2 &ab)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .u32 key;\n\t"
+        "setp.le.s32 p, %2, %6;\n\t"
+        "setp.le.and.s32 p, %3, %7, p;\n\t"
+        "setp.le.and.s32 p, %4, %8, p;\n\t"
+        "setp.le.and.s32 p, %5, %9, p;\n\t"
+        "mad.lo.u32 key, %2, %11, %10;\n\t"
+        "setp.lt.and.u32 p, key, %1, p;\n\t"
+        "@p add.f32 %0, %0, 0f3F800000;\n\t}"
+        : "+f"(cnt)
+        : "r"(t3), "r"(g), "r"(v), "r"(c), "r"(m), "r"(f.x), "r"(f.y), "r"(f.z), "r"(f.w), "r"(ab.x), "r"(ab.y));
+}
+// Packed capacity test: both words are subtracted; a guard bit that fell means some capacity is
+// smaller than the ask. lop3 0x2a = ~(a & b) & c, with the "result != 0" predicate.
+__device__ __forceinline__ void pair_packed(float &cnt, unsigned int t3, unsigned int r0, unsigned int r1,
+                                            unsigned int g, const uint4 &h, unsigned int guards)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, bad;\n\t.reg .u32 d0, d1, e, key;\n\t"
+        "mad.lo.u32 d0, %2, 0xffffffff, %5;\n\t"
+        "mad.lo.u32 d1, %3, 0xffffffff, %6;\n\t"
+        "lop3.and.b32 e|bad, d0, d1, %9, 0x2a, 1;\n\t"
+        "mad.lo.u32 key, %4, %8, %7;\n\t"
+        "setp.lt.and.u32 p, key, %1, !bad;\n\t"
+        "@p add.f32 %0, %0, 0f3F800000;\n\t}"
+        : "+f"(cnt)
+        : "r"(t3), "r"(r0), "r"(r1), "r"(g), "r"(h.x), "r"(h.y), "r"(h.z), "r"(h.w), "r"(guards));
+}
+__device__ __forceinline__ void pair_packed_static(float &cnt, unsigned int t3, unsigned int r0,
+                                                   unsigned int r1, const uint4 &h, unsigned int guards)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, bad;\n\t.reg .u32 d0, d1, e;\n\t"
+        "mad.lo.u32 d0, %2, 0xffffffff, %4;\n\t"
+        "mad.lo.u32 d1, %3, 0xffffffff, %5;\n\t"
+        "lop3.and.b32 e|bad, d0, d1, %7, 0x2a, 1;\n\t"
+        "setp.lt.and.u32 p, %6, %1, !bad;\n\t"
+        "@p add.f32 %0, %0, 0f3F800000;\n\t}"
+        : "+f"(cnt)
+        : "r"(t3), "r"(r0), "r"(r1), "r"(h.x), "r"(h.y), "r"(h.z), "r"(guards));
+}
+
+// Two-mask forms: 0x0c = ~a & b on (d0, guards0); 0xf2 = a | (~b & c) on (e0, d1, guards1).
+__device__ __forceinline__ void pair_packed2(float &cnt, unsigned int t3, unsigned int r0, unsigned int r1,
+                                             unsigned int g, const uint4 &h, unsigned int guards0,
+                                             unsigned int guards1)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, bad;\n\t.reg .u32 d0, d1, e0, e, key;\n\t"
+        "mad.lo.u32 d0, %2, 0xffffffff, %5;\n\t"
+        "mad.lo.u32 d1, %3, 0xffffffff, %6;\n\t"
+        "lop3.b32 e0, d0, %9, 0, 0x0c;\n\t"
+        "lop3.and.b32 e|bad, e0, d1, %10, 0xf2, 1;\n\t"
+        "mad.lo.u32 key, %4, %8, %7;\n\t"
+        "setp.lt.and.u32 p, key, %1, !bad;\n\t"
+        "@p add.f32 %0, %0, 0f3F800000;\n\t}"
+        : "+f"(cnt)
+        : "r"(t3), "r"(r0), "r"(r1), "r"(g), "r"(h.x), "r"(h.y), "r"(h.z), "r"(h.w), "r"(guards0), "r"(guards1));
+}
+__device__ __forceinline__ void pair_packed2_static(float &cnt, unsigned int t3, unsigned int r0,
+                                                    unsigned int r1, const uint4 &h, unsigned int guards0,
+                                                    unsigned int guards1)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, bad;\n\t.reg .u32 d0, d1, e0, e;\n\t"
+        "mad.lo.u32 d0, %2, 0xffffffff, %4;\n\t"
+        "mad.lo.u32 d1, %3, 0xffffffff, %5;\n\t"
+        "lop3.b32 e0, d0, %7, 0, 0x0c;\n\t"
+        "lop3.and.b32 e|bad, e0, d1, %8, 0xf2, 1;\n\t"
+        "setp.lt.and.u32 p, %6, %1, !bad;\n\t"
+        "@p add.f32 %0, %0, 0f3F800000;\n\t}"
+        : "+f"(cnt)
+        : "r"(t3), "r"(r0), "r"(r1), "r"(h.x), "r"(h.y), "r"(h.z), "r"(guards0), "r"(guards1));
+}
+
+template <int MODE> struct ModeTraits {
+    using Key = unsigned int;
+    using Pair = uint2;
+};
+template <> struct ModeTraits<MODE_KEY64> {
+    using Key = unsigned long long;
+    using Pair = ulonglong2;
+};
+
 // ---- one pass: Q requests per group through all tiles of the block's host slice ------------
-template <int Q, int L, typename KeyT>
+template <int Q, int L, int MODE>
 __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *stages,
                                          uint32_t stage_bytes, uint32_t full_bar,
                                          uint32_t empty_bar, volatile unsigned int *abort_flag,
                                          uint32_t &ring_pos, int tile_begin, int tile_end,
-                                         int slice, int n, long long first, int count)
+                                         int slice, long long first, int count)
 {
-    using Pair = typename KeyTraits<KeyT>::Pair;
+    using KeyT = typename ModeTraits<MODE>::Key;
+    using Pair = typename ModeTraits<MODE>::Pair;
     constexpr KeyT kInf = KeyTraits<KeyT>::kInf;
+    constexpr bool kPacked = mode_is_packed(MODE);
     constexpr int kGroups = kComputeThreads / L;
     const int tid = threadIdx.x;
     const int sub = tid % L;
     const int grp = tid / L;
     const int lane = tid & 31;
 
-    int g[Q], v[Q], c[Q], m[Q];
+    // request registers: plain modes keep the four asks, packed modes the two packed words
+    int g[Q], v[kPacked ? 1 : Q], c[kPacked ? 1 : Q], m[kPacked ? 1 : Q];
+    unsigned int r0[kPacked ? Q : 1], r1[kPacked ? Q : 1];
     KeyT t1[Q], t2[Q], t3[Q];
 #pragma unroll
     for (int q = 0; q < Q; ++q) {
         const int idx = q * kGroups + grp;
-        int4 r = make_int4(INT_MAX, 0, 0, 0);
-        if (idx < count) {
-            r = __ldg(p.requests + first + idx);
+        int4 r = make_int4(-1, 0, 0, 0);
+        if (idx < count) r = __ldg(p.requests + first + idx);
+        if (kPacked) {
+            // an ask that is negative or larger than every host's capacity fits nowhere: encode it
+            // as a GPU ask above every host's gmax and keep the other fields inside their widths
+            const bool bad = ((r.x | r.y | r.z | r.w) < 0) | (r.x > p.pack.fmax[0]) | (r.y > p.pack.fmax[1]) |
+                             (r.z > p.pack.fmax[2]) | (r.w > p.pack.fmax[3]);
+            const unsigned int val[4] = {bad ? (unsigned int)p.pack.fmax[0] + 2u : (unsigned int)r.x + 1u,
+                                         bad ? 0u : (unsigned int)r.y, bad ? 0u : (unsigned int)r.z,
+                                         bad ? 0u : (unsigned int)r.w};
+            unsigned int w0 = 0u, w1 = 0u;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const unsigned int piece = val[k] << p.pack.fshift[k];
+                if (p.pack.fword[k]) w1 |= piece; else w0 |= piece;
+            }
+            r0[q] = w0; r1[q] = w1;
+            g[q] = bad ? 0 : r.x;
+        } else {
             if ((r.x | r.y | r.z | r.w) < 0) r.x = INT_MAX;  // a negative ask fits nowhere
+            g[q] = r.x; v[q] = r.y; c[q] = r.z; m[q] = r.w;
         }
-        g[q] = r.x; v[q] = r.y; c[q] = r.z; m[q] = r.w;
         t1[q] = kInf; t2[q] = kInf; t3[q] = kInf;
     }
 
@@ -212,24 +346,90 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
         const uint32_t s = ring_pos % kStages;
         const uint32_t parity = (ring_pos / kStages) & 1u;
         if (!mbar_wait(full_bar + 8u * s, parity, abort_flag)) return false;
-        const int4 *F = reinterpret_cast<const int4 *>(stages + (size_t)s * stage_bytes);
-        const Pair *AB = reinterpret_cast<const Pair *>(stages + (size_t)s * stage_bytes + (size_t)T * 16);
+        const unsigned char *stage = stages + (size_t)s * stage_bytes;
         int hosts = p.Hpad - t * T;
         if (hosts > T) hosts = T;
+        if (MODE == MODE_KEY64) {
+            const int4 *F = reinterpret_cast<const int4 *>(stage);
+            const Pair *AB = reinterpret_cast<const Pair *>(stage + (size_t)T * 16);
 #pragma unroll 2
-        for (int i = sub; i < hosts; i += L) {
-            const int4 f = F[i];
-            const Pair ab = AB[i];
+            for (int i = sub; i < hosts; i += L) {
+                const int4 f = F[i];
+                const Pair ab = AB[i];
 #pragma unroll
-            for (int q = 0; q < Q; ++q) {
-                const bool ok = (g[q] <= f.x) & (v[q] <= f.y) & (c[q] <= f.z) & (m[q] <= f.w);
-                const KeyT key = (KeyT)(unsigned int)g[q] * ab.y + ab.x;
-                if (ok && key < t3[q]) {
-                    t3[q] = max(t2[q], key);
-                    t2[q] = min(t2[q], max(t1[q], key));
-                    t1[q] = min(t1[q], key);
+                for (int q = 0; q < Q; ++q) {
+                    const bool ok = (g[q] <= f.x) & (v[q] <= f.y) & (c[q] <= f.z) & (m[q] <= f.w);
+                    const KeyT key = (KeyT)(unsigned int)g[q] * ab.y + ab.x;
+                    if (ok && key < t3[q]) {
+                        t3[q] = max(t2[q], key);
+                        t2[q] = min(t2[q], max(t1[q], key));
+                        t1[q] = min(t1[q], key);
+                    }
                 }
             }
+        } else if (MODE == MODE_PLAIN) {
+            const int4 *F = reinterpret_cast<const int4 *>(stage);
+            const uint2 *AB = reinterpret_cast<const uint2 *>(stage + (size_t)T * 16);
+            float cnt = 0.f, seen = 0.f;
+            auto chunk = [&](auto width, int i0) {
+                constexpr int W = decltype(width)::value;
+                int4 f[W];
+                uint2 ab[W];
+#pragma unroll
+                for (int u = 0; u < W; ++u) { f[u] = F[i0 + u * L]; ab[u] = AB[i0 + u * L]; }
+#pragma unroll
+                for (int u = 0; u < W; ++u)
+#pragma unroll
+                    for (int q = 0; q < Q; ++q) pair_plain(cnt, (unsigned int)t3[q], g[q], v[q], c[q], m[q], f[u], ab[u]);
+                if (cnt != seen) {  // rare: some request of this lane takes one of these hosts
+                    seen = cnt;
+#pragma unroll
+                    for (int u = 0; u < W; ++u)
+#pragma unroll
+                        for (int q = 0; q < Q; ++q) {
+                            const bool ok = (g[q] <= f[u].x) & (v[q] <= f[u].y) & (c[q] <= f[u].z) & (m[q] <= f[u].w);
+                            const KeyT key = ok ? (KeyT)((unsigned int)g[q] * ab[u].y + ab[u].x) : kInf;
+                            insert3(t1[q], t2[q], t3[q], key);
+                        }
+                }
+            };
+            int i = sub;
+            for (; i + 3 * L < hosts; i += 4 * L) chunk(std::integral_constant<int, 4>{}, i);
+            for (; i < hosts; i += L) chunk(std::integral_constant<int, 1>{}, i);
+        } else {
+            const uint4 *R = reinterpret_cast<const uint4 *>(stage);
+            const unsigned int guards0 = p.pack.guards, guards1 = p.pack.guards1;
+            float cnt = 0.f, seen = 0.f;
+            auto chunk = [&](auto width, int i0) {
+                constexpr int W = decltype(width)::value;
+                uint4 h[W];
+#pragma unroll
+                for (int u = 0; u < W; ++u) h[u] = R[i0 + u * L];
+#pragma unroll
+                for (int u = 0; u < W; ++u)
+#pragma unroll
+                    for (int q = 0; q < Q; ++q) {
+                        if (MODE == MODE_PACKED) pair_packed(cnt, (unsigned int)t3[q], r0[q], r1[q], (unsigned int)g[q], h[u], guards0);
+                        else if (MODE == MODE_PACKED_STATIC) pair_packed_static(cnt, (unsigned int)t3[q], r0[q], r1[q], h[u], guards0);
+                        else if (MODE == MODE_PACKED2) pair_packed2(cnt, (unsigned int)t3[q], r0[q], r1[q], (unsigned int)g[q], h[u], guards0, guards1);
+                        else pair_packed2_static(cnt, (unsigned int)t3[q], r0[q], r1[q], h[u], guards0, guards1);
+                    }
+                if (cnt != seen) {
+                    seen = cnt;
+#pragma unroll
+                    for (int u = 0; u < W; ++u)
+#pragma unroll
+                        for (int q = 0; q < Q; ++q) {
+                            const unsigned int d0 = h[u].x - r0[q], d1 = h[u].y - r1[q];
+                            const bool bad = ((~d0 & guards0) | (~d1 & guards1)) != 0u;
+                            const unsigned int key = mode_is_static(MODE) ? h[u].z : (unsigned int)g[q] * h[u].w + h[u].z;
+                            insert3(t1[q], t2[q], t3[q], (KeyT)(bad ? 0xFFFFFFFFu : key));
+                        }
+                }
+            };
+            int i = sub;
+            for (; i + 3 * L < hosts; i += 4 * L) chunk(std::integral_constant<int, 4>{}, i);
+            for (; i < hosts; i += L) chunk(std::integral_constant<int, 1>{}, i);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty_bar + 8u * s);
@@ -268,17 +468,19 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
             }
         }
     }
-    (void)n;
     return true;
 }
 
-template <int L, typename KeyT, int MAXQ>
-__global__ void __launch_bounds__(kThreads, 2) place_kernel(const __grid_constant__ PlaceParams p)
+template <int L, int MODE>
+__global__ void __launch_bounds__(kThreads, mode_is_static(MODE) ? 3 : 2)
+place_kernel(const __grid_constant__ PlaceParams p)
 {
-    using Pair = typename KeyTraits<KeyT>::Pair;
+    constexpr int MAXQ = mode_max_q(MODE);
+    constexpr int kRecord = mode_record_bytes(MODE);
+    constexpr bool kPacked = mode_is_packed(MODE);
     extern __shared__ __align__(128) unsigned char smem[];
     const int T = p.tile_hosts;
-    const uint32_t stage_bytes = (uint32_t)T * (16u + (uint32_t)sizeof(Pair));
+    const uint32_t stage_bytes = (uint32_t)T * (uint32_t)kRecord;
     unsigned long long *bars = reinterpret_cast<unsigned long long *>(smem + (size_t)kStages * stage_bytes);
     volatile unsigned int *abort_flag = reinterpret_cast<volatile unsigned int *>(bars + 2 * kStages);
     const uint32_t full_bar = smem_addr(bars);
@@ -315,8 +517,7 @@ __global__ void __launch_bounds__(kThreads, 2) place_kernel(const __grid_constan
         uint32_t issued = 0;
         bool ok = true;
         while (ok && passes.next(n, first, count, q)) {
-            const int4 *feas_n = p.feas + (size_t)n * p.Hpad;
-            const Pair *ab_n = reinterpret_cast<const Pair *>(p.ab) + (size_t)n * p.Hpad;
+            const size_t row = (size_t)n * p.Hpad;
             for (int t = tile_begin; t < tile_end; ++t, ++issued) {
                 const uint32_t s = issued % kStages;
                 if (issued >= (uint32_t)kStages) {
@@ -328,12 +529,21 @@ __global__ void __launch_bounds__(kThreads, 2) place_kernel(const __grid_constan
                 }
                 int hosts = p.Hpad - t * T;
                 if (hosts > T) hosts = T;
-                const uint32_t bytes_f = (uint32_t)hosts * 16u;
-                const uint32_t bytes_k = (uint32_t)hosts * (uint32_t)sizeof(Pair);
                 const uint32_t dst = stage0 + s * stage_bytes;
-                mbar_arrive_expect_tx(full_bar + 8u * s, bytes_f + bytes_k);
-                bulk_copy_g2s(dst, feas_n + (size_t)t * T, bytes_f, full_bar + 8u * s);
-                bulk_copy_g2s(dst + (uint32_t)T * 16u, ab_n + (size_t)t * T, bytes_k, full_bar + 8u * s);
+                if (kPacked) {
+                    const uint32_t bytes = (uint32_t)hosts * 16u;
+                    mbar_arrive_expect_tx(full_bar + 8u * s, bytes);
+                    bulk_copy_g2s(dst, p.pk + row + (size_t)t * T, bytes, full_bar + 8u * s);
+                } else {
+                    const uint32_t pair_bytes = (uint32_t)kRecord - 16u;
+                    const uint32_t bytes_f = (uint32_t)hosts * 16u;
+                    const uint32_t bytes_k = (uint32_t)hosts * pair_bytes;
+                    mbar_arrive_expect_tx(full_bar + 8u * s, bytes_f + bytes_k);
+                    bulk_copy_g2s(dst, p.feas + row + (size_t)t * T, bytes_f, full_bar + 8u * s);
+                    bulk_copy_g2s(dst + (uint32_t)T * 16u,
+                                  static_cast<const unsigned char *>(p.ab) + (row + (size_t)t * T) * pair_bytes,
+                                  bytes_k, full_bar + 8u * s);
+                }
             }
         }
         if (!ok) {
@@ -356,8 +566,8 @@ __global__ void __launch_bounds__(kThreads, 2) place_kernel(const __grid_constan
     bool ok = true;
     while (ok && passes.next(n, first, count, q)) {
 #define NBOS_PASS(QV)                                                                         \
-    ok = run_pass<QV, L, KeyT>(p, smem, stage_bytes, full_bar, empty_bar, abort_flag, ring_pos, \
-                               tile_begin, tile_end, slice, n, first, count)
+    ok = run_pass<QV, L, MODE>(p, smem, stage_bytes, full_bar, empty_bar, abort_flag, ring_pos, \
+                               tile_begin, tile_end, slice, first, count)
         if (MAXQ >= 8 && q == 8) NBOS_PASS(8);
         else if (MAXQ >= 4 && q == 4) NBOS_PASS(4);
         else if (MAXQ >= 2 && q == 2) NBOS_PASS(2);
@@ -393,18 +603,59 @@ __global__ void __launch_bounds__(256) merge_kernel(const KeyT *cand, int K, lon
 
 using KernelFn = void (*)(const PlaceParams);
 
-template <typename KeyT, int MAXQ>
-KernelFn pick_kernel(int L)
+template <int MODE>
+KernelFn pick_kernel_l(int L)
 {
     switch (L) {
-        case 1: return place_kernel<1, KeyT, MAXQ>;
-        case 2: return place_kernel<2, KeyT, MAXQ>;
-        case 4: return place_kernel<4, KeyT, MAXQ>;
-        case 8: return place_kernel<8, KeyT, MAXQ>;
-        case 16: return place_kernel<16, KeyT, MAXQ>;
-        case 32: return place_kernel<32, KeyT, MAXQ>;
+        case 1: return place_kernel<1, MODE>;
+        case 2: return place_kernel<2, MODE>;
+        case 4: return place_kernel<4, MODE>;
+        case 8: return place_kernel<8, MODE>;
+        case 16: return place_kernel<16, MODE>;
+        case 32: return place_kernel<32, MODE>;
     }
     return nullptr;
+}
+
+KernelFn pick_kernel(int mode, int L)
+{
+    switch (mode) {
+        case MODE_KEY64: return pick_kernel_l<MODE_KEY64>(L);
+        case MODE_PLAIN: return pick_kernel_l<MODE_PLAIN>(L);
+        case MODE_PACKED: return pick_kernel_l<MODE_PACKED>(L);
+        case MODE_PACKED_STATIC: return pick_kernel_l<MODE_PACKED_STATIC>(L);
+        case MODE_PACKED2: return pick_kernel_l<MODE_PACKED2>(L);
+        case MODE_PACKED2_STATIC: return pick_kernel_l<MODE_PACKED2_STATIC>(L);
+    }
+    return nullptr;
+}
+
+int snapshot_mode(const nbos_snapshot *s, int forced)
+{
+    if (s->key.key_bits == 64) return MODE_KEY64;
+    if (forced == 1 || !s->pack.enabled) return MODE_PLAIN;
+    const bool two = s->pack.guards != s->pack.guards1;
+    if (forced == 2 || !s->key.static_key) return two ? MODE_PACKED2 : MODE_PACKED;
+    return two ? MODE_PACKED2_STATIC : MODE_PACKED_STATIC;
+}
+
+void fill_params(PlaceParams &p, const nbos_snapshot *s, const int32_t *d_requests, int64_t batch,
+                 int32_t *d_out_hosts, int32_t *d_out_found)
+{
+    p.feas = s->d_feas;
+    p.ab = s->d_ab;
+    p.pk = s->d_pk;
+    p.pack = s->pack;
+    p.requests = reinterpret_cast<const int4 *>(d_requests);
+    p.out_hosts = d_out_hosts;
+    p.out_found = d_out_found;
+    p.cand = nullptr;
+    p.status = s->d_status;
+    p.B = batch;
+    p.total = (long long)s->N * batch;
+    p.N = s->N;
+    p.Hpad = s->Hpad;
+    p.id_mask = (1u << s->key.bits_id) - 1u;
 }
 
 bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
@@ -417,33 +668,63 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
 {
     const long long total = (long long)s->N * batch;
     if (total == 0) return NBOS_OK;
-    const bool k64 = s->key.key_bits == 64;
-    const int max_q_kernel = k64 ? 4 : 8;
-    const int pair_bytes = k64 ? 16 : 8;
 
     nbos_launch_config c = {};
     if (cfg) c = *cfg;
-    if (c.reserved[0] | c.reserved[1] | c.reserved[2]) return fail(NBOS_ERR_INVALID_ARG, "launch config: reserved fields must be 0");
+    if (c.reserved[0] | c.reserved[1]) return fail(NBOS_ERR_INVALID_ARG, "launch config: reserved fields must be 0");
     if (c.lanes_per_request && !(is_pow2(c.lanes_per_request) && c.lanes_per_request <= 32))
         return fail(NBOS_ERR_INVALID_ARG, "lanes_per_request must be 1,2,4,8,16 or 32");
     if (c.requests_per_lane && !(is_pow2(c.requests_per_lane) && c.requests_per_lane <= 8))
         return fail(NBOS_ERR_INVALID_ARG, "requests_per_lane must be 1,2,4 or 8");
     if (c.host_split < 0 || c.grid_blocks < 0 || c.tile_hosts < 0 || (c.tile_hosts & 31))
         return fail(NBOS_ERR_INVALID_ARG, "launch config: negative field or tile_hosts not a multiple of 32");
+    if (c.pair_mode < 0 || c.pair_mode > 2)
+        return fail(NBOS_ERR_INVALID_ARG, "pair_mode must be 0 (automatic), 1 (plain compares) or 2 (packed, key computed per pair)");
+
+    const int mode = snapshot_mode(s, c.pair_mode);
+    const bool k64 = mode == MODE_KEY64;
+    const int record = mode_record_bytes(mode);
+    const int max_q_kernel = mode_max_q(mode);
 
     // tile: as many hosts as fit the stage budget, at most the whole (padded) table
     int T = c.tile_hosts ? c.tile_hosts : 1024;
     if (T > s->Hpad) T = s->Hpad;
-    const int max_tile = (64 * 1024) / (16 + pair_bytes) / 32 * 32;  // <= 64 KB per stage
+    const int max_tile = (64 * 1024) / record / 32 * 32;  // <= 64 KB per stage
     if (T > max_tile) T = max_tile;
     const int tiles_total = (s->Hpad + T - 1) / T;
 
-    // lanes per request: as few as still give every SM enough resident threads
-    const long long want_threads = (long long)s->sm_count * 2 * kComputeThreads;
+    KernelFn fn1 = pick_kernel(mode, 1);
+    const size_t smem = (size_t)kStages * T * record + 2 * kStages * 8 + 16;
+    NBOS_CUDA_TRY(cudaFuncSetAttribute(fn1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int per_sm = 0;
+    NBOS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn1, kThreads, smem));
+    if (per_sm < 1) return fail(NBOS_ERR_CUDA, "placement kernel does not fit on an SM (%zu bytes of shared memory)", smem);
+
+    // Lanes per request: estimate, for each L, the pair steps one lane of the busiest block has to
+    // make (passes in units of requests per lane, weighted by how well a pass of that size
+    // amortises the per-host overhead, times hosts per lane) plus the shuffle merges, and take
+    // the cheapest. Large batches end up with few lanes, small ones with a whole warp.
+    const long long want_threads = (long long)s->sm_count * per_sm * kComputeThreads;
     int L = c.lanes_per_request;
     if (!L) {
-        L = 1;
-        while (L < 32 && total * L < want_threads) L <<= 1;
+        const long long slots = (long long)s->sm_count * per_sm;
+        double best = 0.0;
+        for (int cand = 1, lg = 0; cand <= 32; cand <<= 1, ++lg) {
+            const long long groups = kComputeThreads / cand;
+            long long ctas = (total + groups - 1) / groups;
+            if (ctas > slots) ctas = slots;
+            const long long n_req = (total + ctas - 1) / ctas;
+            const long long full = n_req / (groups * max_q_kernel), rem = n_req % (groups * max_q_kernel);
+            int q = max_q_kernel;
+            while (q > 2 && (long long)(q >> 1) * groups >= rem) q >>= 1;
+            const double weight = q >= 8 ? 1.0 : q == 4 ? 1.12 : 1.4;
+            const double units = (double)full * max_q_kernel + (rem ? q * weight : 0.0);
+            const double cost = units * ((double)s->Hpad / cand) + (double)(full + (rem ? 1 : 0)) * lg * max_q_kernel * 4.0;
+            if (cand == 1 || cost < best * 0.98) {
+                best = cost;
+                L = cand;
+            }
+        }
     }
     int K = c.host_split;
     if (!K) {
@@ -459,11 +740,9 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
     int max_q = c.requests_per_lane ? c.requests_per_lane : max_q_kernel;
     if (max_q > max_q_kernel) max_q = max_q_kernel;
 
-    KernelFn fn = k64 ? pick_kernel<unsigned long long, 4>(L) : pick_kernel<unsigned int, 8>(L);
+    KernelFn fn = pick_kernel(mode, L);
     if (!fn) return fail(NBOS_ERR_INVALID_ARG, "no kernel for this launch shape");
-    const size_t smem = (size_t)kStages * T * (16 + pair_bytes) + 2 * kStages * 8 + 16;
     NBOS_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    int per_sm = 0;
     NBOS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kThreads, smem));
     if (per_sm < 1) return fail(NBOS_ERR_CUDA, "placement kernel does not fit on an SM (%zu bytes of shared memory)", smem);
 
@@ -475,22 +754,11 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
     if (req_ctas > cap) req_ctas = cap;
 
     PlaceParams p;
-    p.feas = s->d_feas;
-    p.ab = s->d_ab;
-    p.requests = reinterpret_cast<const int4 *>(d_requests);
-    p.out_hosts = d_out_hosts;
-    p.out_found = d_out_found;
-    p.cand = nullptr;
-    p.status = s->d_status;
-    p.B = batch;
-    p.total = total;
-    p.N = s->N;
-    p.Hpad = s->Hpad;
+    fill_params(p, s, d_requests, batch, d_out_hosts, d_out_found);
     p.tile_hosts = T;
     p.tiles_total = tiles_total;
     p.K = K;
     p.req_ctas = (int)req_ctas;
-    p.id_mask = (1u << s->key.bits_id) - 1u;
     p.max_q = max_q;
 
     if (K > 1) {
@@ -519,7 +787,6 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
     if (e != cudaSuccess) return cuda_fail(e, "placement launch");
     return NBOS_OK;
 }
-
 
 // ---- placement without any allocation ------------------------------------------------------
 // The host-split launch shape needs a candidate buffer (K slices x requests x 3 keys). The
@@ -563,9 +830,10 @@ int launch_place_static(const nbos_snapshot *s, const int32_t *d_requests, int64
     NBOS_CUDA_TRY(cudaGetDevice(&device));
     if (device != s->device)
         return fail(NBOS_ERR_INVALID_ARG, "snapshot was created on device %d, current device is %d", s->device, device);
-    const bool k64 = s->key.key_bits == 64;
+    const int mode = snapshot_mode(s, 0);
+    const bool k64 = mode == MODE_KEY64;
     const int key_bytes = k64 ? 8 : 4;
-    const int pair_bytes = k64 ? 16 : 8;
+    const int record = mode_record_bytes(mode);
 
     // host slices: K tiles-aligned slices of the padded host table
     int K = host_split ? host_split : 4;
@@ -588,8 +856,8 @@ int launch_place_static(const nbos_snapshot *s, const int32_t *d_requests, int64
     if (rc) return rc;
 
     const int L = 32;  // small batches are what this shape is for: one warp per request group
-    KernelFn fn = k64 ? pick_kernel<unsigned long long, 4>(L) : pick_kernel<unsigned int, 8>(L);
-    const size_t smem = (size_t)kStages * T * (16 + pair_bytes) + 2 * kStages * 8 + 16;
+    KernelFn fn = pick_kernel(mode, L);
+    const size_t smem = (size_t)kStages * T * record + 2 * kStages * 8 + 16;
     NBOS_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 0;
     NBOS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kThreads, smem));
@@ -601,23 +869,13 @@ int launch_place_static(const nbos_snapshot *s, const int32_t *d_requests, int64
     if (req_ctas > cap) req_ctas = cap;
 
     PlaceParams p;
-    p.feas = s->d_feas;
-    p.ab = s->d_ab;
-    p.requests = reinterpret_cast<const int4 *>(d_requests);
-    p.out_hosts = d_out_hosts;
-    p.out_found = d_out_found;
+    fill_params(p, s, d_requests, batch, d_out_hosts, d_out_found);
     p.cand = K > 1 ? cand : nullptr;
-    p.status = s->d_status;
-    p.B = batch;
-    p.total = total;
-    p.N = s->N;
-    p.Hpad = s->Hpad;
     p.tile_hosts = T;
     p.tiles_total = tiles_total;
     p.K = K;
     p.req_ctas = (int)req_ctas;
-    p.id_mask = (1u << s->key.bits_id) - 1u;
-    p.max_q = k64 ? 4 : 8;
+    p.max_q = mode_max_q(mode);
 
     // Nothing in the buffer has to start at zero: the placement kernel writes all K * total * 3
     // candidate slots of this call before the merge kernel (next on the stream) reads them.

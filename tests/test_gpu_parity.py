@@ -129,6 +129,76 @@ def test_key_widths_orders_flags(nb, lib_flags, key_order, flags):
             assert_same(got, ref, f"{w.name} order={key_order} flags={flags} lib={lib_flags}")
 
 
+@pytest.mark.parametrize("pair_mode", [0, 1, 2])
+@pytest.mark.parametrize("lanes", [0, 1, 4, 32])
+def test_pair_evaluation_modes(nb, pair_mode, lanes):
+    """Plain compares, packed test with per-pair key, and the automatic choice give the same bytes."""
+    cfg = nb.launch_config(lanes_per_request=lanes, pair_mode=pair_mode)
+    for w in (W.make_config(2, batch=6000), W.mixed_gpu_cluster(900, 2500, seed=31),
+              W.make_config(4, batch=80, n_snapshots=40), W.make_config(3, batch=3000)):
+        for key_order in (0, 1):
+            got, ref = both(nb, w, key_order=key_order, config=cfg)
+            assert_same(got, ref, f"{w.name} pair_mode={pair_mode} lanes={lanes} order={key_order}")
+
+
+def test_packed_test_layouts_and_fallback(nb):
+    """The packed capacity test is used when the four capacities fit two 32-bit words: with one
+    guard mask, with one mask per word, or not at all (plain compares). Same results each way."""
+    w = W.make_config(1, batch=3000)
+    s = nb.snapshot_from_workload(w)
+    info = s.info()
+    assert (info.packed_test, info.static_key, info.presorted) == (1, 1, 1)
+    nb.nbos_snapshot_destroy(s)
+    # memory capacity of exactly 2^20 MB needs 21 bits: 21 + 10 (VRAM) + 2 > 32 -> one mask per word
+    w2 = W.make_config(1, batch=3000)
+    w2.mem_mb[0, 7] = 1 << 20
+    s = nb.snapshot_from_workload(w2)
+    assert s.info().packed_test == 2
+    nb.nbos_snapshot_destroy(s)
+    got, ref = both(nb, w2)
+    assert_same(got, ref, "two guard masks")
+    # capacities far beyond 32 bits in total: plain compares
+    w3 = W.make_config(1, batch=3000)
+    w3.mem_mb[0, 9] = (1 << 31) - 1
+    w3.millicpus[0, 11] = 1 << 30
+    w3.requests[0, :100, 3] = (1 << 31) - 1
+    w3.requests[0, 100:200, 2] = (1 << 30) - 5
+    s = nb.snapshot_from_workload(w3)
+    assert s.info().packed_test == 0
+    nb.nbos_snapshot_destroy(s)
+    got, ref = both(nb, w3)
+    assert_same(got, ref, "plain compares")
+    # mixed GPU counts: the key slope differs between hosts -> not static
+    w4 = W.mixed_gpu_cluster(300, 2000, seed=8)
+    s = nb.snapshot_from_workload(w4)
+    assert s.info().static_key == 0
+    nb.nbos_snapshot_destroy(s)
+    # asks just above and at the largest capacity of each dimension
+    w5 = W.make_config(1, batch=64)
+    for k, arr in enumerate((w5.gpus_total, w5.vram_gb, w5.millicpus, w5.mem_mb)):
+        top = int(arr.max())
+        w5.requests[0, 2 * k] = [1, 16, 1000, 1024]
+        w5.requests[0, 2 * k + 1] = [1, 16, 1000, 1024]
+        w5.requests[0, 2 * k, k] = top
+        w5.requests[0, 2 * k + 1, k] = top + 1
+    got, ref = both(nb, w5)
+    assert_same(got, ref, "asks at the capacity maxima")
+
+
+def test_large_table_is_not_presorted(nb):
+    """More than 8,192 hosts: the table stays in host order; results are the same."""
+    w = W.uniform_cluster(9000, 600, seed=77)
+    s = nb.snapshot_from_workload(w)
+    assert s.info().presorted == 0
+    nb.nbos_snapshot_destroy(s)
+    for shape in (dict(), dict(lanes_per_request=1), dict(lanes_per_request=32, host_split=3)):
+        got, ref = both(nb, w, config=nb.launch_config(**shape) if shape else None)
+        assert_same(got, ref, f"9000 hosts {shape}")
+    w = W.mixed_gpu_cluster(8200, 300, seed=78)
+    got, ref = both(nb, w, key_order=1)
+    assert_same(got, ref, "8200 mixed hosts")
+
+
 def test_key_width_is_chosen_from_the_data(nb):
     w = W.make_config(1)
     s = nb.snapshot_from_workload(w)
