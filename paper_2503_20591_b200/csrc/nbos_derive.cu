@@ -34,29 +34,29 @@ __device__ __forceinline__ int derive_gmax(long long G, long long S, long long C
 }
 
 // grid (blocks_per_snapshot, N). Validates the value ranges and reduces what the key layout
-// depends on. `stats` must be zeroed (g_min preset to INT_MAX) before the launch.
+// depends on. `stats` must be zeroed before the launch (every field is a max- or or-reduction).
 __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
 {
     __shared__ unsigned long long s_mask[16];
     __shared__ unsigned int s_err;
-    __shared__ int s_idle_max, s_g_min;
+    __shared__ int s_idle_max, s_g_min_inv;
     __shared__ unsigned long long s_sub_max;
     __shared__ int s_max4[4];
     const int n = blockIdx.y;
-    if (threadIdx.x < 4) s_max4[threadIdx.x] = threadIdx.x == 0 ? -1 : 0;
+    if (threadIdx.x < 4) s_max4[threadIdx.x] = 0;
     if (threadIdx.x < 16) s_mask[threadIdx.x] = 0ull;
     if (threadIdx.x == 0) {
         s_err = 0u;
         s_idle_max = 0;
-        s_g_min = INT_MAX;
+        s_g_min_inv = 0;
         s_sub_max = 0ull;
     }
     __syncthreads();
     const int2 lim = a.limits[n];
     unsigned int err = 0u;
-    int idle_max = 0, g_min = INT_MAX;
+    int idle_max = 0, g_min_inv = 0;  // INT_MAX - smallest G seen, 0 = none
     unsigned long long sub_max = 0ull;
-    int max_gcap = -1, max_av = 0, max_ac = 0, max_am = 0;
+    int max_gcap1 = 0, max_av = 0, max_ac = 0, max_am = 0;  // max_gcap1 = largest gmax + 1
     for (int h = blockIdx.x * blockDim.x + threadIdx.x; h < a.H; h += gridDim.x * blockDim.x) {
         const size_t i = (size_t)n * a.H + h;
         const int G = a.G[i], S = a.S[i], C = a.C[i];
@@ -66,21 +66,21 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
         if (err) continue;
         if (G >= 1) {
             atomicOr(&s_mask[G >> 6], 1ull << (G & 63));
-            g_min = min(g_min, G);
+            g_min_inv = max(g_min_inv, INT_MAX - G);
         }
         idle_max = max(idle_max, G - C);
         const int gm = derive_gmax(G, S, C, lim.x, lim.y, a.R, a.flags);
         if (gm >= 0) sub_max = max(sub_max, (unsigned long long)S + (unsigned long long)gm);
-        max_gcap = max(max_gcap, gm);
+        max_gcap1 = max(max_gcap1, gm + 1);
         max_av = max(max_av, a.AV[i]);
         max_ac = max(max_ac, a.AC[i]);
         max_am = max(max_am, a.AM[i]);
     }
     if (err) atomicOr(&s_err, err);
     atomicMax(&s_idle_max, idle_max);
-    atomicMin(&s_g_min, g_min);
+    atomicMax(&s_g_min_inv, g_min_inv);
     atomicMax(&s_sub_max, sub_max);
-    atomicMax(&s_max4[0], max_gcap);
+    atomicMax(&s_max4[0], max_gcap1);
     atomicMax(&s_max4[1], max_av);
     atomicMax(&s_max4[2], max_ac);
     atomicMax(&s_max4[3], max_am);
@@ -90,23 +90,12 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
     if (threadIdx.x == 0) {
         if (s_err) atomicOr(&st->err, s_err);
         atomicMax(&st->idle_max, s_idle_max);
-        atomicMin(&st->g_min, s_g_min);
+        atomicMax(&st->g_min_inv, s_g_min_inv);
         atomicMax(&st->sub_max, s_sub_max);
-        atomicMax(&st->max_gcap, s_max4[0]);
+        atomicMax(&st->max_gcap1, s_max4[0]);
         atomicMax(&st->max_av, s_max4[1]);
         atomicMax(&st->max_ac, s_max4[2]);
         atomicMax(&st->max_am, s_max4[3]);
-    }
-}
-
-__global__ void init_stats_kernel(SnapStats *stats, int n)
-{
-    int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n) {
-        SnapStats z = {};
-        z.g_min = INT_MAX;
-        z.max_gcap = -1;
-        stats[i] = z;
     }
 }
 
@@ -122,8 +111,8 @@ struct EmitArgs {
     int bits_idle, bits_sr, bits_id;
 };
 
-constexpr int kSortMaxHosts = 8192;  // largest (padded, power of two) table sorted in shared memory
-constexpr unsigned long long kSortNever = 0xFFFFFFFFFFFFFFFEull;  // hosts that take nothing go last
+constexpr int kSortMaxHosts = 65536;  // larger tables keep host order (ranking is quadratic in the host count)
+constexpr unsigned long long kSortNever = 0xFFFFFFFF00000000ull;  // hosts that take nothing go last (| host index)
 
 // grid (ceil(Hpad / 256), N). One record per (padded) host.
 template <typename KeyT, typename PairT>
@@ -134,7 +123,7 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
     if (h >= a.Hpad) return;
     int4 f = make_int4(-1, 0, 0, 0);  // padding host: takes nothing
     KeyT A = (KeyT)h, B = 0;
-    unsigned long long sk = kSortNever;
+    unsigned long long sk = kSortNever | (unsigned int)h;
     if (h < a.H) {
         const size_t i = (size_t)n * a.H + h;
         const int G = a.G[i], S = a.S[i], C = a.C[i];
@@ -152,7 +141,7 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
                 A = (idle_inv << (a.bits_sr + a.bits_id)) + (sr0 << a.bits_id) + (KeyT)h;
                 B = w << a.bits_id;
             }
-            sk = (unsigned long long)A;
+            sk = sizeof(KeyT) == 4 ? ((unsigned long long)A << 32) | (unsigned int)h : (unsigned long long)A;
         }
     }
     a.sortkey[(size_t)n * a.Hpad + h] = sk;
@@ -163,53 +152,33 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
     reinterpret_cast<PairT *>(a.ab)[(size_t)n * a.Hpad + h] = p;
 }
 
-// Visiting order. One block per snapshot sorts (sortkey, position) in shared memory (bitonic,
-// n2 = power of two >= Hpad) and writes the permutation. Hosts are visited in ascending order of
-// their key at g = 0, which makes later hosts rarely displace an earlier best-three entry.
-__global__ void __launch_bounds__(1024) sort_kernel(const unsigned long long *sortkey, unsigned int *perm,
-                                                    int Hpad, int n2)
+// Visiting order: hosts are visited in ascending order of their key at g = 0 (hosts that take
+// nothing last), which makes later hosts rarely displace an earlier best-three entry. The sort
+// keys are unique, so the position of host i is the number of hosts with a smaller key. Each
+// block counts, for 256 hosts, the smaller keys inside one chunk of kRankChunk keys staged in
+// shared memory, and adds its partial count to rank[i]. grid (ceil(Hpad/256), ceil(Hpad/chunk), N).
+constexpr int kRankChunk = 1024;
+__global__ void __launch_bounds__(256) rank_kernel(const unsigned long long *sortkey, unsigned int *rank, int Hpad)
 {
-    extern __shared__ __align__(16) unsigned char sort_smem[];
-    unsigned long long *keys = reinterpret_cast<unsigned long long *>(sort_smem);
-    unsigned int *pos = reinterpret_cast<unsigned int *>(sort_smem + (size_t)n2 * 8);
-    const size_t base = (size_t)blockIdx.x * Hpad;
-    for (int i = threadIdx.x; i < n2; i += blockDim.x) {
-        keys[i] = i < Hpad ? sortkey[base + i] : 0xFFFFFFFFFFFFFFFFull;
-        pos[i] = (unsigned int)i;
-    }
+    __shared__ unsigned long long chunk[kRankChunk];
+    const size_t base = (size_t)blockIdx.z * Hpad;
+    const int j0 = blockIdx.y * kRankChunk;
+    const int nj = min(kRankChunk, Hpad - j0);
+    for (int j = threadIdx.x; j < nj; j += blockDim.x) chunk[j] = sortkey[base + j0 + j];
     __syncthreads();
-    for (int k = 2; k <= n2; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int i = threadIdx.x; i < n2; i += blockDim.x) {
-                const int other = i ^ j;
-                if (other > i) {
-                    const bool up = (i & k) == 0;
-                    const unsigned long long a = keys[i], b = keys[other];
-                    if ((a > b) == up) {
-                        keys[i] = b;
-                        keys[other] = a;
-                        const unsigned int t = pos[i];
-                        pos[i] = pos[other];
-                        pos[other] = t;
-                    }
-                }
-            }
-            __syncthreads();
-        }
-    }
-    for (int i = threadIdx.x; i < Hpad; i += blockDim.x) perm[base + i] = pos[i];
-}
-
-__global__ void identity_perm_kernel(unsigned int *perm, int Hpad, size_t total)
-{
-    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < total) perm[i] = (unsigned int)(i % Hpad);
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= Hpad) return;
+    const unsigned long long ki = sortkey[base + i];
+    unsigned int smaller = 0;
+#pragma unroll 8
+    for (int j = 0; j < nj; ++j) smaller += chunk[j] < ki ? 1u : 0u;
+    if (smaller) atomicAdd(&rank[base + i], smaller);
 }
 
 struct FinalizeArgs {
     const int4 *tmp_feas;
     const void *tmp_ab;
-    const unsigned int *perm;
+    const unsigned int *rank;   // position of each host in visiting order, or null = host order
     int4 *feas;
     void *ab;
     uint4 *pk;
@@ -217,14 +186,14 @@ struct FinalizeArgs {
     PackLayout pack;
 };
 
-// grid (ceil(Hpad / 256), N): gather the records into visiting order and build the packed form.
+// grid (ceil(Hpad / 256), N): move the records into visiting order and build the packed form.
 template <typename PairT>
 __global__ void __launch_bounds__(256) finalize_kernel(const FinalizeArgs a)
 {
-    const int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= a.Hpad) return;
+    const int src = blockIdx.x * blockDim.x + threadIdx.x;
+    if (src >= a.Hpad) return;
     const size_t base = (size_t)blockIdx.y * a.Hpad;
-    const unsigned int src = a.perm[base + j];
+    const unsigned int j = a.rank ? a.rank[base + src] : (unsigned int)src;
     const int4 f = a.tmp_feas[base + src];
     const PairT p = reinterpret_cast<const PairT *>(a.tmp_ab)[base + src];
     a.feas[base + j] = f;
@@ -303,10 +272,10 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     if (!h_limits || !h_stats || !h_lambda) return fail(NBOS_ERR_NO_MEMORY, "host allocation failed");
     for (int n = 0; n < N; ++n) h_limits[n] = make_int2(d->limit_num[n], d->limit_den[n]);
 
-    NBOS_CUDA_TRY(cudaMemsetAsync(ws + lay.off_status, 0, 256, stream));
+    // status word, limits, lambda and scan statistics are contiguous: one clear
+    NBOS_CUDA_TRY(cudaMemsetAsync(ws + lay.off_status, 0, lay.off_feas - lay.off_status, stream));
     NBOS_CUDA_TRY(cudaMemcpyAsync(d_limits, h_limits, sizeof(int2) * (size_t)N,
                                   cudaMemcpyHostToDevice, stream));
-    init_stats_kernel<<<(N + 255) / 256, 256, 0, stream>>>(d_stats, N);
 
     ScanArgs sa{d_G, d_S, d_C, d_AV, d_AC, d_AM, d_limits, d_stats, H, s->R, s->flags};
     int bx = (H + 255) / 256;
@@ -336,8 +305,8 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
         }
         h_lambda[n] = (long long)lambda;
         if (st.idle_max > idle_max) idle_max = st.idle_max;
-        if (st.g_min != INT_MAX) {
-            const unsigned long long w_max = lambda / (unsigned long long)st.g_min;
+        if (st.g_min_inv != 0) {
+            const unsigned long long w_max = lambda / (unsigned long long)(INT_MAX - st.g_min_inv);
             if (st.sub_max > (1ull << 62) / (w_max ? w_max : 1))
                 return fail(NBOS_ERR_RANGE, "snapshot %d: subscription values too large for a 63-bit key", n);
             const unsigned long long m = st.sub_max * w_max;
@@ -358,7 +327,7 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
         int distinct_g = 0;
         for (int w = 0; w < 16; ++w) distinct_g += __builtin_popcountll(st.g_mask[w]);
         if (distinct_g > 1) k.static_key = 0;
-        if (st.max_gcap > fmax[0]) fmax[0] = st.max_gcap;
+        if (st.max_gcap1 - 1 > fmax[0]) fmax[0] = st.max_gcap1 - 1;
         if (st.max_av > fmax[1]) fmax[1] = st.max_av;
         if (st.max_ac > fmax[2]) fmax[2] = st.max_ac;
         if (st.max_am > fmax[3]) fmax[3] = st.max_am;
@@ -408,20 +377,13 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     NBOS_CUDA_TRY(cudaGetLastError());
 
     // visiting order
-    int n2 = 32;
-    while (n2 < Hpad) n2 <<= 1;
-    s->presorted = n2 <= kSortMaxHosts;
+    s->presorted = Hpad <= kSortMaxHosts;
     if (s->presorted) {
-        const size_t sort_smem = (size_t)n2 * 12;
-        NBOS_CUDA_TRY(cudaFuncSetAttribute(sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sort_smem));
-        const int sort_threads = n2 / 2 > 1024 ? 1024 : n2 / 2 < 32 ? 32 : n2 / 2;
-        sort_kernel<<<N, sort_threads, sort_smem, stream>>>(sortkey, perm, Hpad, n2);
-    } else {
-        const size_t total = (size_t)N * Hpad;
-        identity_perm_kernel<<<(unsigned int)((total + 255) / 256), 256, 0, stream>>>(perm, Hpad, total);
+        NBOS_CUDA_TRY(cudaMemsetAsync(perm, 0, sizeof(unsigned int) * (size_t)N * Hpad, stream));
+        rank_kernel<<<dim3((Hpad + 255) / 256, (Hpad + kRankChunk - 1) / kRankChunk, N), 256, 0, stream>>>(sortkey, perm, Hpad);
+        NBOS_CUDA_TRY(cudaGetLastError());
     }
-    NBOS_CUDA_TRY(cudaGetLastError());
-    FinalizeArgs fa{tmp_feas, tmp_ab, perm, reinterpret_cast<int4 *>(ws + lay.off_feas), ws + lay.off_ab,
+    FinalizeArgs fa{tmp_feas, tmp_ab, s->presorted ? perm : nullptr, reinterpret_cast<int4 *>(ws + lay.off_feas), ws + lay.off_ab,
                     reinterpret_cast<uint4 *>(ws + lay.off_pk), Hpad, pk};
     if (k.key_bits == 32)
         finalize_kernel<uint2><<<grid, 256, 0, stream>>>(fa);

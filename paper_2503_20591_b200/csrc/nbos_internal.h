@@ -24,10 +24,10 @@ int cuda_fail(cudaError_t e, const char *what);
 struct SnapStats {                 // one per snapshot, filled by the scan kernel
     unsigned int err;              // bit mask of ERR_* below
     int idle_max;                  // max over hosts of G - C
-    int g_min;                     // min over hosts with G >= 1 of G (INT_MAX if none)
+    int g_min_inv;                 // INT_MAX - (min over hosts with G >= 1 of G); 0 if none
     int pad;
     unsigned long long sub_max;    // max over hosts that can take something of S + gmax
-    int max_gcap, max_av, max_ac, max_am;  // maxima of gmax and of the three capacities
+    int max_gcap1, max_av, max_ac, max_am;  // maxima of gmax + 1 and of the three capacities
     unsigned long long g_mask[16]; // bit G set if some host has G GPUs (G in 1..1023)
 };
 enum : unsigned int {

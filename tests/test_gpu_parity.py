@@ -185,11 +185,12 @@ def test_packed_test_layouts_and_fallback(nb):
     assert_same(got, ref, "asks at the capacity maxima")
 
 
-def test_large_table_is_not_presorted(nb):
-    """More than 8,192 hosts: the table stays in host order; results are the same."""
+def test_large_tables(nb):
+    """Up to 65,536 hosts the table is stored in key order; beyond that it stays in host order.
+    Results are the same either way."""
     w = W.uniform_cluster(9000, 600, seed=77)
     s = nb.snapshot_from_workload(w)
-    assert s.info().presorted == 0
+    assert s.info().presorted == 1
     nb.nbos_snapshot_destroy(s)
     for shape in (dict(), dict(lanes_per_request=1), dict(lanes_per_request=32, host_split=3)):
         got, ref = both(nb, w, config=nb.launch_config(**shape) if shape else None)
@@ -197,6 +198,13 @@ def test_large_table_is_not_presorted(nb):
     w = W.mixed_gpu_cluster(8200, 300, seed=78)
     got, ref = both(nb, w, key_order=1)
     assert_same(got, ref, "8200 mixed hosts")
+    w = W.uniform_cluster(70000, 48, seed=79)
+    s = nb.snapshot_from_workload(w)
+    assert s.info().presorted == 0
+    nb.nbos_snapshot_destroy(s)
+    for shape in (dict(), dict(lanes_per_request=1)):
+        got, ref = both(nb, w, config=nb.launch_config(**shape) if shape else None)
+        assert_same(got, ref, f"70000 hosts {shape}")
 
 
 def test_key_width_is_chosen_from_the_data(nb):
