@@ -6,6 +6,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 
 #include "nbos_internal.h"
@@ -78,6 +79,34 @@ int check_device(int *device, int *sm_count)
     return NBOS_OK;
 }
 
+// Side streams and events used by nbos_place_batch_host, one set per device, created on first use.
+struct HostPipe {
+    static constexpr int kStreams = 3;
+    std::mutex mutex;
+    bool ready = false;
+    cudaStream_t streams[kStreams] = {};
+    cudaEvent_t start = nullptr, done[kStreams] = {};
+};
+HostPipe g_pipes[64];
+std::mutex g_pipes_mutex;
+
+int host_pipe(int device, HostPipe **out)
+{
+    if (device < 0 || device >= 64) return fail(NBOS_ERR_INVALID_ARG, "device index %d not supported", device);
+    std::lock_guard<std::mutex> lock(g_pipes_mutex);
+    HostPipe &p = g_pipes[device];
+    if (!p.ready) {
+        for (int j = 0; j < HostPipe::kStreams; ++j) {
+            NBOS_CUDA_TRY(cudaStreamCreateWithFlags(&p.streams[j], cudaStreamNonBlocking));
+            NBOS_CUDA_TRY(cudaEventCreateWithFlags(&p.done[j], cudaEventDisableTiming));
+        }
+        NBOS_CUDA_TRY(cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming));
+        p.ready = true;
+    }
+    *out = &p;
+    return NBOS_OK;
+}
+
 nbos_snapshot *new_handle(const nbos_snapshot_desc *d)
 {
     nbos_snapshot *s = new (std::nothrow) nbos_snapshot();
@@ -89,6 +118,7 @@ nbos_snapshot *new_handle(const nbos_snapshot_desc *d)
     s->key_order = d->key_order;
     s->flags = d->flags;
     s->owns_workspace = false;
+    s->owner_stream = nullptr;
     return s;
 }
 
@@ -157,22 +187,23 @@ int nbos_snapshot_create_host(const nbos_snapshot_desc *desc, void *cuda_stream,
     const size_t arr_bytes = (cells * sizeof(int32_t) + 255) & ~(size_t)255;
     const size_t need = workspace_layout(desc->n_snapshots, pad_hosts(desc->n_hosts)).total;
     void *ws = nullptr, *staging = nullptr;
-    cudaError_t e = cudaMalloc(&ws, need);
-    if (e == cudaSuccess) e = cudaMalloc(&staging, 6 * arr_bytes);
+    cudaError_t e = cudaMallocAsync(&ws, need, stream);
+    if (e == cudaSuccess) e = cudaMallocAsync(&staging, 6 * arr_bytes, stream);
     if (e != cudaSuccess) {
-        cudaFree(ws);
+        if (ws) cudaFreeAsync(ws, stream);
         cudaGetLastError();
-        return fail(NBOS_ERR_NO_MEMORY, "cudaMalloc failed: %s", cudaGetErrorString(e));
+        return fail(NBOS_ERR_NO_MEMORY, "device allocation failed: %s", cudaGetErrorString(e));
     }
     nbos_snapshot *s = new_handle(desc);
     if (!s) {
-        cudaFree(ws);
-        cudaFree(staging);
+        cudaFreeAsync(ws, stream);
+        cudaFreeAsync(staging, stream);
         return fail(NBOS_ERR_NO_MEMORY, "host allocation failed");
     }
     s->workspace = ws;
     s->workspace_bytes = need;
     s->owns_workspace = true;
+    s->owner_stream = stream;
     s->device = device;
     s->sm_count = sms;
     const int32_t *src[6] = {desc->gpus_total, desc->gpus_subscribed, desc->gpus_committed,
@@ -185,13 +216,9 @@ int nbos_snapshot_create_host(const nbos_snapshot_desc *desc, void *cuda_stream,
     }
     rc = e == cudaSuccess ? derive_snapshot(s, desc, dev[0], dev[1], dev[2], dev[3], dev[4], dev[5], stream)
                           : cuda_fail(e, "copying host-state arrays to the device");
-    if (rc == NBOS_OK) {
-        e = cudaStreamSynchronize(stream);  // the staging buffer is released next
-        if (e != cudaSuccess) rc = cuda_fail(e, "cudaStreamSynchronize");
-    }
-    cudaFree(staging);
+    cudaFreeAsync(staging, stream);  // stream-ordered: after the kernels that read it
     if (rc) {
-        cudaFree(ws);
+        cudaFreeAsync(ws, stream);
         delete s;
         return rc;
     }
@@ -204,8 +231,8 @@ int nbos_snapshot_destroy(nbos_snapshot *snap)
     if (!snap) return NBOS_OK;
     int rc = NBOS_OK;
     if (snap->owns_workspace) {
-        cudaError_t e = cudaFree(snap->workspace);
-        if (e != cudaSuccess) rc = cuda_fail(e, "cudaFree");
+        cudaError_t e = cudaFreeAsync(snap->workspace, nullptr);  // legacy default stream: ordered after blocking streams
+        if (e != cudaSuccess) rc = cuda_fail(e, "cudaFreeAsync");
     }
     delete snap;
     return rc;
@@ -264,9 +291,17 @@ int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_hos
     if (batch_per_snapshot == 0) return NBOS_OK;
     if (!requests_host || !out_hosts_host) return fail(NBOS_ERR_INVALID_ARG, "requests / out_hosts is NULL");
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const size_t total = (size_t)snap->N * (size_t)batch_per_snapshot;
-    const size_t req_bytes = total * 16, out_bytes = total * 12, found_bytes = out_found_host ? total * 4 : 0;
+    const long long total = (long long)snap->N * batch_per_snapshot;
+    const size_t req_bytes = (size_t)total * 16, out_bytes = (size_t)total * 12,
+                 found_bytes = out_found_host ? (size_t)total * 4 : 0;
     auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+
+    // side streams for the copy / compute overlap, created once per process and device
+    HostPipe *pipe = nullptr;
+    int rc = host_pipe(snap->device, &pipe);
+    if (rc) return rc;
+    std::lock_guard<std::mutex> lock(pipe->mutex);
+
     char *buf = nullptr;
     cudaError_t e = cudaMallocAsync(reinterpret_cast<void **>(&buf), up(req_bytes) + up(out_bytes) + up(found_bytes), stream);
     if (e != cudaSuccess) {
@@ -276,13 +311,34 @@ int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_hos
     int32_t *d_req = reinterpret_cast<int32_t *>(buf);
     int32_t *d_out = reinterpret_cast<int32_t *>(buf + up(req_bytes));
     int32_t *d_found = out_found_host ? reinterpret_cast<int32_t *>(buf + up(req_bytes) + up(out_bytes)) : nullptr;
-    int rc = NBOS_OK;
-    e = cudaMemcpyAsync(d_req, requests_host, req_bytes, cudaMemcpyHostToDevice, stream);
-    if (e == cudaSuccess) {
-        rc = launch_place(snap, d_req, batch_per_snapshot, d_out, d_found, stream, nullptr);
-        if (rc == NBOS_OK) e = cudaMemcpyAsync(out_hosts_host, d_out, out_bytes, cudaMemcpyDeviceToHost, stream);
-        if (rc == NBOS_OK && e == cudaSuccess && d_found)
-            e = cudaMemcpyAsync(out_found_host, d_found, found_bytes, cudaMemcpyDeviceToHost, stream);
+
+    // chunks of the flattened request list: copy in, place, copy out, round-robin over the side
+    // streams so that the copies of one chunk overlap the kernel of another
+    long long n_chunks = total / (128 * 1024);
+    if (n_chunks < 1) n_chunks = 1;
+    if (n_chunks > 16) n_chunks = 16;
+    const long long chunk = ((total + n_chunks - 1) / n_chunks + 31) & ~31ll;
+    e = cudaEventRecord(pipe->start, stream);
+    for (int j = 0; j < HostPipe::kStreams && e == cudaSuccess; ++j) e = cudaStreamWaitEvent(pipe->streams[j], pipe->start, 0);
+    int used = 0;
+    for (long long lo = 0, i = 0; lo < total && e == cudaSuccess && rc == NBOS_OK; lo += chunk, ++i) {
+        const long long n = total - lo < chunk ? total - lo : chunk;
+        cudaStream_t st = pipe->streams[i % HostPipe::kStreams];
+        if (i < HostPipe::kStreams) used = (int)i + 1;
+        e = cudaMemcpyAsync(d_req + lo * 4, requests_host + lo * 4, (size_t)n * 16, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) break;
+        rc = launch_place(snap, d_req, batch_per_snapshot, d_out, d_found, st, nullptr, lo, n);
+        if (rc) break;
+        e = cudaMemcpyAsync(out_hosts_host + lo * 3, d_out + lo * 3, (size_t)n * 12, cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess && d_found)
+            e = cudaMemcpyAsync(out_found_host + lo, d_found + lo, (size_t)n * 4, cudaMemcpyDeviceToHost, st);
+    }
+    // join the side streams back into the caller's stream (also on the error paths, so that the
+    // staging buffer is not released under work that was already queued)
+    for (int j = 0; j < used; ++j) {
+        cudaError_t e3 = cudaEventRecord(pipe->done[j], pipe->streams[j]);
+        if (e3 == cudaSuccess) e3 = cudaStreamWaitEvent(stream, pipe->done[j], 0);
+        if (e3 != cudaSuccess && e == cudaSuccess) e = e3;
     }
     cudaFreeAsync(buf, stream);
     cudaError_t e2 = cudaStreamSynchronize(stream);

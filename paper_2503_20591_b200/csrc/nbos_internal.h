@@ -79,6 +79,7 @@ struct nbos_snapshot {
     nbos::PackLayout pack;
     int presorted;
     int device, sm_count;
+    cudaStream_t owner_stream;  // stream the owned workspace was allocated on (create_host)
 };
 
 namespace nbos {
@@ -88,10 +89,12 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *host_desc, const
                     const int32_t *d_S, const int32_t *d_C, const int32_t *d_AV,
                     const int32_t *d_AC, const int32_t *d_AM, cudaStream_t stream);
 
-// a1-a9: the placement launch (nbos_place.cu).
+// a1-a9: the placement launch (nbos_place.cu). The pointers are those of the whole batch; the
+// launch handles the flattened requests [range_first, range_first + range_count) of the N * batch
+// (range_count < 0: all that follow range_first).
 int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batch,
                  int32_t *d_out_hosts, int32_t *d_out_found, cudaStream_t stream,
-                 const nbos_launch_config *cfg);
+                 const nbos_launch_config *cfg, long long range_first = 0, long long range_count = -1);
 
 // Host-split placement whose candidate buffer is a fixed array inside the module (no allocation).
 int launch_place_static(const nbos_snapshot *s, const int32_t *d_requests, int64_t batch,

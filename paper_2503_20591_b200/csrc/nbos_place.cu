@@ -63,6 +63,7 @@ struct PlaceParams {
     void *cand;             // [K][N * B][3] keys, only when K > 1
     unsigned int *status;
     long long B, total;     // requests per snapshot, N * B
+    long long first_req, n_req;  // this launch handles flattened requests [first_req, first_req + n_req)
     int N, Hpad;
     int tile_hosts, tiles_total, K, req_ctas;
     unsigned int id_mask;
@@ -191,11 +192,13 @@ __device__ __forceinline__ void block_request_range(const PlaceParams &p, int cr
                                                     long long &hi)
 {
     // split in units of 32 requests so that a warp's 128-bit loads start on a 512-byte line
-    const long long units = (p.total + 31) >> 5;
+    const long long units = (p.n_req + 31) >> 5;
     lo = (units * cr / p.req_ctas) << 5;
     hi = (units * (cr + 1) / p.req_ctas) << 5;
-    if (lo > p.total) lo = p.total;
-    if (hi > p.total) hi = p.total;
+    if (lo > p.n_req) lo = p.n_req;
+    if (hi > p.n_req) hi = p.n_req;
+    lo += p.first_req;
+    hi += p.first_req;
 }
 
 // ---- the pair step --------------------------------------------------------------------------
@@ -456,7 +459,7 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
             if (idx >= count) continue;
             const long long r = first + idx;
             if (p.K > 1) {
-                KeyT *cand = reinterpret_cast<KeyT *>(p.cand) + ((long long)slice * p.total + r) * 3;
+                KeyT *cand = reinterpret_cast<KeyT *>(p.cand) + ((long long)slice * p.n_req + (r - p.first_req)) * 3;
                 cand[0] = t1[q]; cand[1] = t2[q]; cand[2] = t3[q];
             } else {
                 int32_t *o = p.out_hosts + r * 3;
@@ -580,15 +583,16 @@ place_kernel(const __grid_constant__ PlaceParams p)
 // a7: merge the K per-slice candidate triples of each request.
 template <typename KeyT>
 __global__ void __launch_bounds__(256) merge_kernel(const KeyT *cand, int K, long long total,
-                                                    unsigned int id_mask, int32_t *out_hosts,
-                                                    int32_t *out_found)
+                                                    long long first_req, unsigned int id_mask,
+                                                    int32_t *out_hosts, int32_t *out_found)
 {
     constexpr KeyT kInf = KeyTraits<KeyT>::kInf;
-    for (long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x; r < total;
-         r += (long long)gridDim.x * blockDim.x) {
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        const long long r = first_req + i;
         KeyT t1 = kInf, t2 = kInf, t3 = kInf;
         for (int k = 0; k < K; ++k) {
-            const KeyT *c = cand + ((long long)k * total + r) * 3;
+            const KeyT *c = cand + ((long long)k * total + i) * 3;
             insert3(t1, t2, t3, c[0]);
             insert3(t1, t2, t3, c[1]);
             insert3(t1, t2, t3, c[2]);
@@ -653,6 +657,8 @@ void fill_params(PlaceParams &p, const nbos_snapshot *s, const int32_t *d_reques
     p.status = s->d_status;
     p.B = batch;
     p.total = (long long)s->N * batch;
+    p.first_req = 0;
+    p.n_req = p.total;
     p.N = s->N;
     p.Hpad = s->Hpad;
     p.id_mask = (1u << s->key.bits_id) - 1u;
@@ -664,10 +670,11 @@ bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
 
 int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batch,
                  int32_t *d_out_hosts, int32_t *d_out_found, cudaStream_t stream,
-                 const nbos_launch_config *cfg)
+                 const nbos_launch_config *cfg, long long range_first, long long range_count)
 {
-    const long long total = (long long)s->N * batch;
-    if (total == 0) return NBOS_OK;
+    if (range_count < 0) range_count = (long long)s->N * batch - range_first;
+    const long long total = range_count;  // requests of this launch
+    if (total <= 0) return NBOS_OK;
 
     nbos_launch_config c = {};
     if (cfg) c = *cfg;
@@ -755,6 +762,8 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
 
     PlaceParams p;
     fill_params(p, s, d_requests, batch, d_out_hosts, d_out_found);
+    p.first_req = range_first;
+    p.n_req = range_count;
     p.tile_hosts = T;
     p.tiles_total = tiles_total;
     p.K = K;
@@ -777,10 +786,10 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
         if (blocks > (long long)s->sm_count * 8) blocks = (long long)s->sm_count * 8;
         if (k64)
             merge_kernel<unsigned long long><<<(unsigned int)blocks, 256, 0, stream>>>(
-                static_cast<const unsigned long long *>(p.cand), K, total, p.id_mask, d_out_hosts, d_out_found);
+                static_cast<const unsigned long long *>(p.cand), K, total, p.first_req, p.id_mask, d_out_hosts, d_out_found);
         else
             merge_kernel<unsigned int><<<(unsigned int)blocks, 256, 0, stream>>>(
-                static_cast<const unsigned int *>(p.cand), K, total, p.id_mask, d_out_hosts, d_out_found);
+                static_cast<const unsigned int *>(p.cand), K, total, p.first_req, p.id_mask, d_out_hosts, d_out_found);
         e = cudaGetLastError();
     }
     if (p.cand) cudaFreeAsync(p.cand, stream);
@@ -886,10 +895,10 @@ int launch_place_static(const nbos_snapshot *s, const int32_t *d_requests, int64
         if (blocks > (long long)s->sm_count * 8) blocks = (long long)s->sm_count * 8;
         if (k64)
             merge_kernel<unsigned long long><<<(unsigned int)blocks, 256, 0, stream>>>(
-                static_cast<const unsigned long long *>(cand), K, total, p.id_mask, d_out_hosts, d_out_found);
+                static_cast<const unsigned long long *>(cand), K, total, p.first_req, p.id_mask, d_out_hosts, d_out_found);
         else
             merge_kernel<unsigned int><<<(unsigned int)blocks, 256, 0, stream>>>(
-                static_cast<const unsigned int *>(cand), K, total, p.id_mask, d_out_hosts, d_out_found);
+                static_cast<const unsigned int *>(cand), K, total, p.first_req, p.id_mask, d_out_hosts, d_out_found);
         NBOS_CUDA_TRY(cudaGetLastError());
     }
     return NBOS_OK;
