@@ -35,7 +35,7 @@ ALGORITHMIC_OPS_PER_PAIR = 6      # 4 capacity compares + 1 multiply-add (key) +
 L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (read + write) of one placement-kernel launch on the default workload, from the ncu
 # capture summarised under profiles/. None while no capture matches the current kernel.
-PLACE_KERNEL_DRAM_BYTES_PER_LAUNCH = None
+PLACE_KERNEL_DRAM_BYTES_PER_LAUNCH = 16_914_176  # profiles/place_kernel_cfg3_launch_list.md
 
 
 def parse_args():
@@ -50,6 +50,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-sample", type=int, default=None, help="requests in the CPU sample")
+    ap.add_argument("--lanes", type=int, default=0,
+                    help="force lanes per request (profiling a shrunk batch in the full batch's shape)")
     return ap.parse_args()
 
 
@@ -212,6 +214,7 @@ def run_ours(args):
     workspace = torch.empty(nb.nbos_snapshot_workspace_bytes(w.n_snapshots, w.n_hosts),
                             dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
+    launch_cfg = nb.launch_config(lanes_per_request=args.lanes) if args.lanes else None
 
     def step(i, ev=None):
         snap = nb.nbos_snapshot_create(w.n_snapshots, w.n_hosts, lim_num, lim_den, *d_state,
@@ -219,7 +222,7 @@ def run_ours(args):
         k = i % n_rot
         if ev is not None:
             ev[0].record(stream)
-        nb.nbos_place_batch(snap, d_req[k], d_out[k], d_found[k], stream=stream)
+        nb.nbos_place_batch(snap, d_req[k], d_out[k], d_found[k], stream=stream, config=launch_cfg)
         if ev is not None:
             ev[1].record(stream)
         return snap
@@ -329,7 +332,8 @@ def run_ours(args):
                 "when all hosts share the key slope), so frac_of_alu_pipe_alone can exceed 1",
         "ops_per_pair": ALGORITHMIC_OPS_PER_PAIR, "kernel_ms": kern_ms,
         "pairs_per_s_kernel": w.pairs / (kern_ms * 1e-3),
-        "traffic": PLACE_KERNEL_DRAM_BYTES_PER_LAUNCH,
+        "traffic": PLACE_KERNEL_DRAM_BYTES_PER_LAUNCH if (args.workload == 3 and args.batch is None) else None,
+        "algorithmic_bytes": w.decisions * (16 + 12 + 4),
         "stream_gbs": w.decisions * (16 + 12 + 4) / (kern_ms * 1e-3) / 1e9,
         "probe_alu_gops": probe["alu_gops"], "probe_imad_gops": probe["imad_gops"],
         "probe_both_gops": probe["both_gops"],
