@@ -13,5 +13,6 @@ from .placement import (  # noqa: F401
     place,
     place_workload,
     ranks_before,
+    select_executors,
     subscription_ratio,
 )

@@ -155,3 +155,62 @@ int nbos_oracle_place(const nbos_oracle_cluster *cl, const int32_t *requests, in
     free(taken);
     return 0;
 }
+
+/*
+ * Executor selection for a cell execution (Section 3.2.2). The scheduler looks at the servers
+ * that host the kernel's three replicas. A replica whose server lacks the resources to run the
+ * cell now is told to yield; when the scheduler has the resource information it designates the
+ * executor itself. If all three must yield, the election fails and a replica has to migrate
+ * (Section 3.2.3).
+ *
+ * "Can run now" = the server has the idle resources to bind at once: g <= G - C idle GPUs, and
+ * the three other asks within the capacities passed in (the caller passes what is idle). The SR
+ * limit is not tested here: the replica is already subscribed on its server.
+ * Reading where the paper is silent: among the replicas that can run, the designated executor is
+ * the first in the default policy's order (Section 3.4.1): more idle GPUs, then lower current
+ * SR = S / (G * R), then lower host index, then lower replica slot.
+ *
+ *   requests       [n_kernels][4]  (GPUs, VRAM GB, millicpus, memory MB)
+ *   replica_hosts  [n_kernels][3]  host index of each replica, -1 = no such replica
+ *   out_executor   [n_kernels]     host index of the designated executor, -1 = all yield
+ *   out_can_run    [n_kernels]     bit k set: replica k could run now
+ */
+int nbos_oracle_select_executors(const nbos_oracle_cluster *cl, const int32_t *requests,
+                                 const int32_t *replica_hosts, int64_t n_kernels,
+                                 int32_t *out_executor, int32_t *out_can_run)
+{
+    if (!cl || n_kernels < 0 || cl->replicas_R < 1) return -1;
+    for (int64_t k = 0; k < n_kernels; ++k) {
+        int32_t g = requests[4 * k + 0], v = requests[4 * k + 1];
+        int32_t c = requests[4 * k + 2], m = requests[4 * k + 3];
+        int32_t best = -1, mask = 0;
+        for (int slot = 0; slot < 3; ++slot) {
+            int32_t h = replica_hosts[3 * k + slot];
+            if (h < 0 || h >= cl->n_hosts) continue;
+            int64_t G = cl->G[h], C = cl->C[h];
+            if (g < 0 || v < 0 || c < 0 || m < 0) continue;
+            if (G < 1) continue;
+            if ((int64_t)g > G - C) continue;          /* idle GPUs, bound at once */
+            if (v > cl->AV[h] || c > cl->AC[h] || m > cl->AM[h]) continue;
+            mask |= 1 << slot;
+            if (best < 0) {
+                best = h;
+                continue;
+            }
+            /* does h come before the current best? */
+            int64_t idle_h = G - C, idle_b = (int64_t)cl->G[best] - cl->C[best];
+            int before;
+            if (idle_h != idle_b) {
+                before = idle_h > idle_b;
+            } else {
+                int sr = nbos_oracle_compare_sr_after(cl->S[h], cl->G[h], cl->S[best], cl->G[best], 0,
+                                                      cl->replicas_R);
+                before = sr != 0 ? sr < 0 : h < best;   /* equal host: keep the earlier slot */
+            }
+            if (before) best = h;
+        }
+        out_executor[k] = best;
+        out_can_run[k] = mask;
+    }
+    return 0;
+}

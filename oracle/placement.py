@@ -65,6 +65,9 @@ def _load():
         lib.nbos_oracle_place.restype = ctypes.c_int
         lib.nbos_oracle_place.argtypes = [ctypes.POINTER(_Cluster), _i32p, ctypes.c_int64,
                                           _i32p, _i32p]
+        lib.nbos_oracle_select_executors.restype = ctypes.c_int
+        lib.nbos_oracle_select_executors.argtypes = [ctypes.POINTER(_Cluster), _i32p, _i32p,
+                                                     ctypes.c_int64, _i32p, _i32p]
         _lib = lib
     return _lib
 
@@ -116,6 +119,25 @@ def place(G, S, C, AV, AC, AM, limit_num, limit_den, requests, replicas_R=3,
     if rc != 0:
         raise ValueError("nbos_oracle_place rejected its arguments")
     return hosts, found
+
+
+def select_executors(G, S, C, AV, AC, AM, requests, replica_hosts, replicas_R=3):
+    """Section 3.2.2: which replica of each kernel runs the cell. Returns (executor [M] int32
+    host index or -1, can_run [M] int32 bit mask over the three replica slots)."""
+    cl, keep = _cluster(G, S, C, AV, AC, AM, 1, 1, replicas_R, 0, 0)
+    req = _as_i32(requests).reshape(-1, 4)
+    rep = _as_i32(replica_hosts).reshape(-1, 3)
+    if rep.shape[0] != req.shape[0]:
+        raise ValueError("one row of replica hosts per request")
+    m = req.shape[0]
+    ex = np.empty((m,), dtype=np.int32)
+    mask = np.empty((m,), dtype=np.int32)
+    rc = _load().nbos_oracle_select_executors(ctypes.byref(cl), req.ctypes.data_as(_i32p),
+                                              rep.ctypes.data_as(_i32p), m,
+                                              ex.ctypes.data_as(_i32p), mask.ctypes.data_as(_i32p))
+    if rc != 0:
+        raise ValueError("nbos_oracle_select_executors rejected its arguments")
+    return ex, mask
 
 
 def place_workload(w, key_order=KEY_IDLE_FIRST, flags=0, threads: int = 1,
