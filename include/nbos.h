@@ -239,6 +239,41 @@ int nbos_place_batch_noalloc(const nbos_snapshot *snap, const int32_t *requests,
                              int64_t batch_per_snapshot, int32_t *out_hosts, int32_t *out_found,
                              void *cuda_stream, int32_t host_split);
 
+/*
+ * Executor selection for a batch of cell executions (Section 3.2.2). When a cell is submitted,
+ * the scheduler looks at the servers hosting the kernel's three replicas: a replica whose server
+ * lacks the resources to run the cell now is told to yield, and with the resource information at
+ * hand the scheduler designates the executor itself; if all three must yield, a replica has to
+ * migrate (Section 3.2.3 -- find the target with nbos_place_batch on a snapshot created with
+ * NBOS_REQUIRE_IDLE_GPUS and the idle capacities; its first column is the best target).
+ *
+ *   can run now   <=>  g,v,c,m >= 0 and G >= 1 and g <= G - C and v <= vram_gb and c <= millicpus
+ *                      and m <= mem_mb  (pass the idle capacities). The SR limit is not tested:
+ *                      the replica is already subscribed on its server.
+ *   designated    =    among the replicas that can run, the first by (G - C descending,
+ *                      S / (G * R) ascending -- compared exactly --, host index ascending, replica
+ *                      slot ascending). The paper does not say which runnable replica is picked;
+ *                      this is the default placement policy's order (Section 3.4.1).
+ *
+ *   state          DEVICE arrays [n_hosts] int32 of one cluster snapshot (not validated; a host
+ *                  index outside 0..n_hosts-1 in replica_hosts, e.g. -1, means "no such replica")
+ *   requests       DEVICE [n_kernels * 4] int32, 16-byte aligned: GPUs, VRAM GB, millicpus, MB
+ *   replica_hosts  DEVICE [n_kernels * 3] int32
+ *   out_executor   DEVICE [n_kernels] int32: host index of the designated executor, -1 = all yield
+ *   out_can_run    DEVICE [n_kernels] int32: bit k set = the replica in slot k can run now
+ * Asynchronous on `cuda_stream`. Errors: INVALID_ARG, CUDA, UNSUPPORTED_DEVICE.
+ */
+typedef struct nbos_cluster_state {
+    int32_t n_hosts;
+    int32_t replicas_R;
+    const int32_t *gpus_total, *gpus_subscribed, *gpus_committed;
+    const int32_t *vram_gb, *millicpus, *mem_mb;
+} nbos_cluster_state;
+
+int nbos_select_executors(const nbos_cluster_state *state, const int32_t *requests,
+                          const int32_t *replica_hosts, int64_t n_kernels, int32_t *out_executor,
+                          int32_t *out_can_run, void *cuda_stream);
+
 /* Synchronises `cuda_stream` and returns the sticky device status of this snapshot: NBOS_OK, or
  * NBOS_ERR_DEVICE_TIMEOUT if some kernel gave up on a bounded wait (its outputs are then
  * undefined). */

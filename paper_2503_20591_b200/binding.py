@@ -36,7 +36,8 @@ NBOS_PROBE_MIX_BOTH = 2
 EXPORTED_SYMBOLS = (
     "nbos_snapshot_workspace_bytes", "nbos_snapshot_create", "nbos_snapshot_create_host",
     "nbos_snapshot_destroy", "nbos_snapshot_get_info", "nbos_place_batch", "nbos_place_batch_ex",
-    "nbos_place_batch_host", "nbos_place_batch_noalloc", "nbos_snapshot_status", "nbos_strerror", "nbos_last_error_detail",
+    "nbos_place_batch_host", "nbos_place_batch_noalloc", "nbos_select_executors",
+    "nbos_snapshot_status", "nbos_strerror", "nbos_last_error_detail",
     "nbos_probe_int32_issue", "nbos_probe_wait_timeout",
 )
 
@@ -64,6 +65,15 @@ class nbos_snapshot_info(ctypes.Structure):
         ("packed_test", ctypes.c_int32), ("static_key", ctypes.c_int32),
         ("presorted", ctypes.c_int32), ("reserved", ctypes.c_int32),
         ("workspace_bytes", ctypes.c_int64),
+    ]
+
+
+class nbos_cluster_state(ctypes.Structure):
+    _fields_ = [
+        ("n_hosts", ctypes.c_int32), ("replicas_R", ctypes.c_int32),
+        ("gpus_total", ctypes.c_void_p), ("gpus_subscribed", ctypes.c_void_p),
+        ("gpus_committed", ctypes.c_void_p), ("vram_gb", ctypes.c_void_p),
+        ("millicpus", ctypes.c_void_p), ("mem_mb", ctypes.c_void_p),
     ]
 
 
@@ -106,6 +116,7 @@ def load_library() -> ctypes.CDLL:
     lib.nbos_place_batch_ex.argtypes = [vp, vp, i64, vp, vp, vp, P(nbos_launch_config)]
     lib.nbos_place_batch_host.argtypes = [vp, vp, i64, vp, vp, vp]
     lib.nbos_place_batch_noalloc.argtypes = [vp, vp, i64, vp, vp, vp, ctypes.c_int32]
+    lib.nbos_select_executors.argtypes = [P(nbos_cluster_state), vp, vp, i64, vp, vp, vp]
     lib.nbos_snapshot_status.argtypes = [vp, vp]
     lib.nbos_strerror.argtypes = [ctypes.c_int]
     lib.nbos_strerror.restype = ctypes.c_char_p
@@ -311,6 +322,30 @@ def nbos_place_batch_noalloc(snap: Snapshot, requests, out_hosts, out_found=None
         raise ValueError("out_found must hold n_snapshots * batch values")
     _check(lib.nbos_place_batch_noalloc(snap.handle, _ptr(requests), b, _ptr(out_hosts),
                                         _ptr(out_found), _stream_ptr(stream), host_split))
+
+
+def nbos_select_executors(gpus_total, gpus_subscribed, gpus_committed, vram_gb, millicpus, mem_mb,
+                          requests, replica_hosts, out_executor, out_can_run, replicas_R=3,
+                          stream=None) -> None:
+    """Device tensors: six state arrays [H], requests [M,4], replica_hosts [M,3], outputs [M]."""
+    lib = load_library()
+    arrs = [_i32(a, n, "cuda") for n, a in zip(("gpus_total", "gpus_subscribed", "gpus_committed",
+                                                "vram_gb", "millicpus", "mem_mb"),
+                                               (gpus_total, gpus_subscribed, gpus_committed, vram_gb,
+                                                millicpus, mem_mb))]
+    h = arrs[0].numel()
+    if any(a.numel() != h for a in arrs):
+        raise ValueError("the six cluster-state arrays must have the same length")
+    for n, t in (("requests", requests), ("replica_hosts", replica_hosts),
+                 ("out_executor", out_executor), ("out_can_run", out_can_run)):
+        _i32(t, n, "cuda")
+    m = requests.numel() // 4
+    if requests.numel() != 4 * m or replica_hosts.numel() != 3 * m or out_executor.numel() != m \
+            or out_can_run.numel() != m:
+        raise ValueError("requests [M,4], replica_hosts [M,3], outputs [M] must agree on M")
+    st = nbos_cluster_state(h, replicas_R, *[_ptr(a) for a in arrs])
+    _check(lib.nbos_select_executors(ctypes.byref(st), _ptr(requests), _ptr(replica_hosts), m,
+                                     _ptr(out_executor), _ptr(out_can_run), _stream_ptr(stream)))
 
 
 def nbos_probe_int32_issue(mix: int, iters: int, blocks: int, threads: int, stream=None):

@@ -1,0 +1,115 @@
+"""GPU parity for executor selection (Section 3.2.2) and the execute -> migrate flow
+(Section 3.2.3), against the CPU checker, bit-exact."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2503_20591_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def nb():
+    import torch
+    from paper_2503_20591_b200 import binding, build as lib_build
+    lib_build.build()
+    assert torch.cuda.is_available()
+    binding.load_library()
+    return binding
+
+
+def draw_kernels(rng, w, m):
+    """m kernels with three distinct replica hosts each and a cell that asks for idle resources."""
+    h = w.n_hosts
+    rep = np.stack([rng.choice(h, size=3, replace=False) for _ in range(m)]).astype(np.int32)
+    g = rng.integers(0, 9, size=m)
+    req = np.stack([g, 16 * g, rng.integers(1000, 16001, size=m), rng.integers(1024, 65537, size=m)],
+                   axis=1).astype(np.int32)
+    return req, rep
+
+
+def gpu_select(nb, w, req, rep):
+    import torch
+    dev = [torch.from_numpy(getattr(w, k)[0]).cuda() for k in w.HOST_FIELDS]
+    ex = torch.full((req.shape[0],), -9, dtype=torch.int32, device="cuda")
+    mask = torch.full((req.shape[0],), -9, dtype=torch.int32, device="cuda")
+    nb.nbos_select_executors(*dev, torch.from_numpy(req).cuda(), torch.from_numpy(rep).cuda(), ex, mask,
+                             replicas_R=w.replicas_R)
+    torch.cuda.synchronize()
+    return ex.cpu().numpy(), mask.cpu().numpy()
+
+
+def cpu_select(w, req, rep):
+    return oracle.select_executors(*[getattr(w, k)[0] for k in w.HOST_FIELDS], req, rep,
+                                   replicas_R=w.replicas_R)
+
+
+@pytest.mark.parametrize("maker", [lambda: W.make_config(1), lambda: W.make_config(2),
+                                   lambda: W.mixed_gpu_cluster(500, 16, seed=5),
+                                   lambda: W.uniform_cluster(3, 16, seed=6)])
+@pytest.mark.parametrize("m", [1, 1000, 300_001])
+def test_executor_selection_matches_the_checker(nb, maker, m):
+    w = maker()
+    rng = np.random.default_rng(m)
+    req, rep = draw_kernels(rng, w, m)
+    rep[rng.random(m) < 0.03, rng.integers(0, 3)] = -1          # missing replicas
+    req[rng.random(m) < 0.01, 0] = -1                           # nonsense asks
+    if m > 10:
+        rep[5] = [0, 0, 0]                                       # degenerate: same host three times
+        rep[6] = [w.n_hosts, -5, 1 << 30]                        # out-of-range ids are "no replica"
+    got = gpu_select(nb, w, req, rep)
+    ref = cpu_select(w, req, rep)
+    np.testing.assert_array_equal(got[0], ref[0])
+    np.testing.assert_array_equal(got[1], ref[1])
+    if m >= 1000:
+        assert (ref[0] >= 0).any()
+
+
+def test_execute_then_migrate_flow(nb):
+    """Kernels whose three replicas must all yield get a migration target: the best host of the
+    idle-resources placement (first column). That target is never one of the yielding hosts."""
+    import torch
+    w = W.make_config(2)                     # heavily loaded cluster: many failed elections
+    rng = np.random.default_rng(3)
+    m = 50_000
+    req, rep = draw_kernels(rng, w, m)
+    ex, mask = gpu_select(nb, w, req, rep)
+    ref_ex, ref_mask = cpu_select(w, req, rep)
+    np.testing.assert_array_equal(ex, ref_ex)
+    failed = np.nonzero(ex < 0)[0]
+    assert failed.size > 100 and failed.size < m
+    # migration targets for the failed elections
+    snap = nb.snapshot_from_workload(w, flags=nb.NBOS_REQUIRE_IDLE_GPUS)
+    mig_req = np.ascontiguousarray(req[failed])[None]
+    out = torch.empty((1, failed.size, 3), dtype=torch.int32, device="cuda")
+    found = torch.empty((1, failed.size), dtype=torch.int32, device="cuda")
+    nb.nbos_place_batch(snap, torch.from_numpy(mig_req).cuda(), out, found)
+    assert nb.nbos_snapshot_status(snap) == nb.NBOS_OK
+    nb.nbos_snapshot_destroy(snap)
+    target = out.cpu().numpy()[0, :, 0]
+    ref_hosts, _ = oracle.place(*[getattr(w, k)[0] for k in w.HOST_FIELDS], int(w.limit_num[0]),
+                                int(w.limit_den[0]), mig_req[0], replicas_R=w.replicas_R,
+                                flags=oracle.REQUIRE_IDLE_GPUS)
+    np.testing.assert_array_equal(target, ref_hosts[:, 0])
+    has_target = target >= 0
+    assert has_target.any()
+    # a host that made its replica yield cannot be the target (it lacks the idle resources)
+    assert not (target[has_target, None] == rep[failed][has_target]).any()
+
+
+def test_argument_errors(nb):
+    import torch
+    w = W.make_config(0)
+    dev = [torch.from_numpy(getattr(w, k)[0]).cuda() for k in w.HOST_FIELDS]
+    req = torch.zeros((4, 4), dtype=torch.int32, device="cuda")
+    rep = torch.zeros((4, 3), dtype=torch.int32, device="cuda")
+    out = torch.zeros((4,), dtype=torch.int32, device="cuda")
+    with pytest.raises(ValueError):
+        nb.nbos_select_executors(*dev, req, rep[:3], out, out)
+    with pytest.raises(nb.NbosError) as e:
+        nb.nbos_select_executors(*dev, req, rep, out, out, replicas_R=0)
+    assert e.value.status == nb.NBOS_ERR_INVALID_ARG
+    nb.nbos_select_executors(*dev, req[:0], rep[:0], out[:0], out[:0])   # empty batch is a no-op
