@@ -7,12 +7,16 @@ from .placement import (  # noqa: F401
     KEY_IDLE_FIRST,
     KEY_SR_FIRST,
     REQUIRE_IDLE_GPUS,
+    autoscale,
     build,
+    cluster_limit,
+    cluster_sums,
     compare_sr_after,
     feasible,
     place,
     place_workload,
     ranks_before,
+    scale_out_deficit,
     select_executors,
     subscription_ratio,
 )

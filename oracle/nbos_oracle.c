@@ -214,3 +214,56 @@ int nbos_oracle_select_executors(const nbos_oracle_cluster *cl, const int32_t *r
     }
     return 0;
 }
+
+/*
+ * Cluster-wide quantities of Sections 3.4.1 and 3.4.2.
+ *   sums[0] = sum of G (GPUs of all servers), sums[1] = sum of S (subscribed GPUs),
+ *   sums[2] = sum of C (GPUs in active use).
+ */
+void nbos_oracle_cluster_sums(const nbos_oracle_cluster *cl, int64_t *sums)
+{
+    sums[0] = sums[1] = sums[2] = 0;
+    for (int32_t h = 0; h < cl->n_hosts; ++h) {
+        sums[0] += cl->G[h];
+        sums[1] += cl->S[h];
+        sums[2] += cl->C[h];
+    }
+}
+
+/* Section 3.4.1, third factor: the dynamic cluster-wide SR limit is sum(S) / (sum(G) * R).
+ * Returned as the rational num / den. den = 0 when the cluster has no GPUs (then no server is a
+ * candidate anyway and the caller must not place against it). */
+void nbos_oracle_cluster_limit(const nbos_oracle_cluster *cl, int64_t *num, int64_t *den)
+{
+    int64_t sums[3];
+    nbos_oracle_cluster_sums(cl, sums);
+    *num = sums[1];
+    *den = sums[0] * cl->replicas_R;
+}
+
+/* Section 3.4.2: the expected capacity is f * sum(C), f = f_num / f_den (the paper uses 1.05).
+ * +1: current capacity sum(G) is smaller than that -> scale out.
+ * -1: the expected capacity is smaller than what is provisioned -> servers may be released.
+ *  0: equal. Exact integer comparison. */
+int nbos_oracle_autoscale(int64_t sum_G, int64_t sum_C, int64_t f_num, int64_t f_den)
+{
+    int64_t expected_scaled = f_num * sum_C; /* f * sum(C) * f_den */
+    int64_t have_scaled = f_den * sum_G;
+    return (have_scaled < expected_scaled) - (expected_scaled < have_scaled);
+}
+
+/* Sections 3.2.1 / 3.4.2: a kernel for which fewer than three servers were found needs
+ * "however many additional servers are required". deficit = sum of (3 - found),
+ * short_requests = number of requests with found < 3. */
+void nbos_oracle_scale_out_deficit(const int32_t *found, int64_t batch, int64_t *deficit,
+                                   int64_t *short_requests)
+{
+    *deficit = 0;
+    *short_requests = 0;
+    for (int64_t r = 0; r < batch; ++r) {
+        if (found[r] < NBOS_ORACLE_REPLICAS_PLACED) {
+            *deficit += NBOS_ORACLE_REPLICAS_PLACED - found[r];
+            *short_requests += 1;
+        }
+    }
+}

@@ -68,6 +68,15 @@ def _load():
         lib.nbos_oracle_select_executors.restype = ctypes.c_int
         lib.nbos_oracle_select_executors.argtypes = [ctypes.POINTER(_Cluster), _i32p, _i32p,
                                                      ctypes.c_int64, _i32p, _i32p]
+        i64p = ctypes.POINTER(ctypes.c_int64)
+        lib.nbos_oracle_cluster_sums.restype = None
+        lib.nbos_oracle_cluster_sums.argtypes = [ctypes.POINTER(_Cluster), i64p]
+        lib.nbos_oracle_cluster_limit.restype = None
+        lib.nbos_oracle_cluster_limit.argtypes = [ctypes.POINTER(_Cluster), i64p, i64p]
+        lib.nbos_oracle_autoscale.restype = ctypes.c_int
+        lib.nbos_oracle_autoscale.argtypes = [ctypes.c_int64] * 4
+        lib.nbos_oracle_scale_out_deficit.restype = None
+        lib.nbos_oracle_scale_out_deficit.argtypes = [_i32p, ctypes.c_int64, i64p, i64p]
         _lib = lib
     return _lib
 
@@ -138,6 +147,38 @@ def select_executors(G, S, C, AV, AC, AM, requests, replica_hosts, replicas_R=3)
     if rc != 0:
         raise ValueError("nbos_oracle_select_executors rejected its arguments")
     return ex, mask
+
+
+def cluster_sums(G, S, C, replicas_R=3):
+    """(sum G, sum S, sum C) of one snapshot."""
+    z = np.zeros(len(G), dtype=np.int32)
+    cl, keep = _cluster(G, S, C, z, z, z, 1, 1, replicas_R, 0, 0)
+    out = (ctypes.c_int64 * 3)()
+    _load().nbos_oracle_cluster_sums(ctypes.byref(cl), out)
+    return int(out[0]), int(out[1]), int(out[2])
+
+
+def cluster_limit(G, S, C, replicas_R=3):
+    """Dynamic cluster-wide SR limit of Section 3.4.1 as (num, den) = (sum S, sum G * R)."""
+    z = np.zeros(len(G), dtype=np.int32)
+    cl, keep = _cluster(G, S, C, z, z, z, 1, 1, replicas_R, 0, 0)
+    num, den = ctypes.c_int64(0), ctypes.c_int64(0)
+    _load().nbos_oracle_cluster_limit(ctypes.byref(cl), ctypes.byref(num), ctypes.byref(den))
+    return int(num.value), int(den.value)
+
+
+def autoscale(sum_G, sum_C, f_num=21, f_den=20) -> int:
+    """Section 3.4.2 with f = f_num / f_den: +1 scale out, -1 may release servers, 0 equal."""
+    return int(_load().nbos_oracle_autoscale(int(sum_G), int(sum_C), int(f_num), int(f_den)))
+
+
+def scale_out_deficit(found):
+    """(sum of 3 - found, number of requests with found < 3) over one batch."""
+    f = _as_i32(found).reshape(-1)
+    d, n = ctypes.c_int64(0), ctypes.c_int64(0)
+    _load().nbos_oracle_scale_out_deficit(f.ctypes.data_as(_i32p), f.shape[0], ctypes.byref(d),
+                                          ctypes.byref(n))
+    return int(d.value), int(n.value)
 
 
 def place_workload(w, key_order=KEY_IDLE_FIRST, flags=0, threads: int = 1,
