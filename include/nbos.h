@@ -65,6 +65,10 @@ extern "C" {
 /* flags */
 #define NBOS_REQUIRE_IDLE_GPUS 1 /* Section 3.2.3: also require g <= G - C                   */
 #define NBOS_FORCE_KEY64 2       /* build the 64-bit key table even if 32 bits would do      */
+#define NBOS_LIMIT_CLUSTER_SR 4  /* Section 3.4.1, third factor: ignore limit_num / limit_den (they may
+                                  * be NULL) and use each snapshot's own cluster-wide SR,
+                                  * sum(S) / (sum(G) * R), as its limit. An empty cluster (sum S = 0)
+                                  * then admits only g = 0; the paper gives no floor.          */
 
 #define NBOS_MAX_HOSTS (1 << 20)   /* per snapshot                          */
 #define NBOS_MAX_GPUS_PER_HOST 1023
@@ -89,7 +93,7 @@ typedef struct nbos_snapshot_desc {
     int32_t n_hosts;     /* 1 <= H <= NBOS_MAX_HOSTS                  */
     int32_t replicas_R;  /* 1 .. NBOS_MAX_REPLICAS; the paper uses 3  */
     int32_t key_order;   /* NBOS_KEY_*                                */
-    int32_t flags;       /* NBOS_REQUIRE_IDLE_GPUS | NBOS_FORCE_KEY64 */
+    int32_t flags;       /* NBOS_REQUIRE_IDLE_GPUS | NBOS_FORCE_KEY64 | NBOS_LIMIT_CLUSTER_SR */
     int32_t reserved;    /* must be 0                                 */
     const int32_t *limit_num; /* HOST [N] in both create variants     */
     const int32_t *limit_den; /* HOST [N]                             */
@@ -273,6 +277,32 @@ typedef struct nbos_cluster_state {
 int nbos_select_executors(const nbos_cluster_state *state, const int32_t *requests,
                           const int32_t *replica_hosts, int64_t n_kernels, int32_t *out_executor,
                           int32_t *out_can_run, void *cuda_stream);
+
+/*
+ * Cluster sums and the auto-scaler rule (Sections 3.4.1, 3.4.2), per snapshot:
+ *   out_sums[4n + 0] = sum of G   (GPUs provisioned)
+ *   out_sums[4n + 1] = sum of S   (GPUs subscribed; sum S / (sum G * R) is the cluster-wide SR)
+ *   out_sums[4n + 2] = sum of C   (GPUs in active use)
+ *   out_sums[4n + 3] = +1 if sum G < f * sum C   (capacity below the expected f * sum C: scale out)
+ *                      -1 if f * sum C < sum G   (more provisioned than expected: servers may go)
+ *                       0 if equal;   f = f_num / f_den, compared exactly (the paper uses 1.05 = 21/20)
+ * Arrays: DEVICE [n_snapshots * n_hosts] int32 (not validated); out_sums: DEVICE [n_snapshots * 4]
+ * int64. Asynchronous on `cuda_stream`.
+ */
+int nbos_cluster_sums(const int32_t *gpus_total, const int32_t *gpus_subscribed,
+                      const int32_t *gpus_committed, int32_t n_snapshots, int32_t n_hosts,
+                      int32_t f_num, int32_t f_den, int64_t *out_sums, void *cuda_stream);
+
+/*
+ * Scale-out deficit of a placed batch (Sections 3.2.1, 3.4.2: when fewer than three candidate
+ * servers exist, "however many additional servers are required" are provisioned), per snapshot:
+ *   out_deficit[2n + 0] = sum over the batch of (3 - found)
+ *   out_deficit[2n + 1] = number of requests with found < 3
+ * found: DEVICE [n_snapshots * batch_per_snapshot] int32 as written by nbos_place_batch;
+ * out_deficit: DEVICE [n_snapshots * 2] int64. Asynchronous on `cuda_stream`.
+ */
+int nbos_scale_out_deficit(const int32_t *found, int32_t n_snapshots, int64_t batch_per_snapshot,
+                           int64_t *out_deficit, void *cuda_stream);
 
 /* Synchronises `cuda_stream` and returns the sticky device status of this snapshot: NBOS_OK, or
  * NBOS_ERR_DEVICE_TIMEOUT if some kernel gave up on a bounded wait (its outputs are then

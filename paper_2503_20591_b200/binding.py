@@ -27,6 +27,7 @@ NBOS_KEY_IDLE_FIRST = 0
 NBOS_KEY_SR_FIRST = 1
 NBOS_REQUIRE_IDLE_GPUS = 1
 NBOS_FORCE_KEY64 = 2
+NBOS_LIMIT_CLUSTER_SR = 4
 
 NBOS_PROBE_MIX_ALU = 0
 NBOS_PROBE_MIX_IMAD = 1
@@ -37,6 +38,7 @@ EXPORTED_SYMBOLS = (
     "nbos_snapshot_workspace_bytes", "nbos_snapshot_create", "nbos_snapshot_create_host",
     "nbos_snapshot_destroy", "nbos_snapshot_get_info", "nbos_place_batch", "nbos_place_batch_ex",
     "nbos_place_batch_host", "nbos_place_batch_noalloc", "nbos_select_executors",
+    "nbos_cluster_sums", "nbos_scale_out_deficit",
     "nbos_snapshot_status", "nbos_strerror", "nbos_last_error_detail",
     "nbos_probe_int32_issue", "nbos_probe_wait_timeout",
 )
@@ -117,6 +119,8 @@ def load_library() -> ctypes.CDLL:
     lib.nbos_place_batch_host.argtypes = [vp, vp, i64, vp, vp, vp]
     lib.nbos_place_batch_noalloc.argtypes = [vp, vp, i64, vp, vp, vp, ctypes.c_int32]
     lib.nbos_select_executors.argtypes = [P(nbos_cluster_state), vp, vp, i64, vp, vp, vp]
+    lib.nbos_cluster_sums.argtypes = [vp, vp, vp] + [ctypes.c_int32] * 4 + [vp, vp]
+    lib.nbos_scale_out_deficit.argtypes = [vp, ctypes.c_int32, i64, vp, vp]
     lib.nbos_snapshot_status.argtypes = [vp, vp]
     lib.nbos_strerror.argtypes = [ctypes.c_int]
     lib.nbos_strerror.restype = ctypes.c_char_p
@@ -181,10 +185,13 @@ class Snapshot:
 
 def _make_desc(n_snapshots, n_hosts, replicas_R, key_order, flags, limit_num, limit_den, arrays,
                device_type):
-    ln = _i32(limit_num, "limit_num", "cpu")
-    ld = _i32(limit_den, "limit_den", "cpu")
-    if ln.numel() != n_snapshots or ld.numel() != n_snapshots:
-        raise ValueError("limit_num / limit_den need one entry per snapshot")
+    if flags & NBOS_LIMIT_CLUSTER_SR and limit_num is None:
+        ln = ld = None
+    else:
+        ln = _i32(limit_num, "limit_num", "cpu")
+        ld = _i32(limit_den, "limit_den", "cpu")
+        if ln.numel() != n_snapshots or ld.numel() != n_snapshots:
+            raise ValueError("limit_num / limit_den need one entry per snapshot")
     arrs = []
     for name, a in zip(("gpus_total", "gpus_subscribed", "gpus_committed", "vram_gb", "millicpus",
                         "mem_mb"), arrays):
@@ -348,6 +355,32 @@ def nbos_select_executors(gpus_total, gpus_subscribed, gpus_committed, vram_gb, 
                                      _ptr(out_executor), _ptr(out_can_run), _stream_ptr(stream)))
 
 
+def nbos_cluster_sums(gpus_total, gpus_subscribed, gpus_committed, n_snapshots, n_hosts, out_sums,
+                      f_num=21, f_den=20, stream=None) -> None:
+    """Device tensors [N*H] int32 in; out_sums [N,4] int64 = (sum G, sum S, sum C, auto-scaler sign)."""
+    for n, t in (("gpus_total", gpus_total), ("gpus_subscribed", gpus_subscribed),
+                 ("gpus_committed", gpus_committed)):
+        _i32(t, n, "cuda")
+        if t.numel() != n_snapshots * n_hosts:
+            raise ValueError(f"{n} must have n_snapshots * n_hosts elements")
+    if out_sums.dtype != torch.int64 or out_sums.numel() != 4 * n_snapshots or not out_sums.is_cuda:
+        raise ValueError("out_sums must be a CUDA int64 tensor of n_snapshots * 4 elements")
+    _check(load_library().nbos_cluster_sums(_ptr(gpus_total), _ptr(gpus_subscribed), _ptr(gpus_committed),
+                                            n_snapshots, n_hosts, f_num, f_den, _ptr(out_sums),
+                                            _stream_ptr(stream)))
+
+
+def nbos_scale_out_deficit(found, n_snapshots, out_deficit, stream=None) -> None:
+    """found [N,B] int32 (CUDA) in; out_deficit [N,2] int64 = (sum of 3 - found, requests short)."""
+    _i32(found, "found", "cuda")
+    if found.numel() % n_snapshots:
+        raise ValueError("found must hold n_snapshots * batch values")
+    if out_deficit.dtype != torch.int64 or out_deficit.numel() != 2 * n_snapshots or not out_deficit.is_cuda:
+        raise ValueError("out_deficit must be a CUDA int64 tensor of n_snapshots * 2 elements")
+    _check(load_library().nbos_scale_out_deficit(_ptr(found), n_snapshots, found.numel() // n_snapshots,
+                                                 _ptr(out_deficit), _stream_ptr(stream)))
+
+
 def nbos_probe_int32_issue(mix: int, iters: int, blocks: int, threads: int, stream=None):
     """Returns (thread-level integer instructions, milliseconds)."""
     ops, ms = ctypes.c_double(0), ctypes.c_float(0)
@@ -378,8 +411,9 @@ def snapshot_from_workload(w, device="cuda", key_order=NBOS_KEY_IDLE_FIRST, flag
                            stream=None) -> Snapshot:
     """Copy a generated workload's host state to the device and create a snapshot from it."""
     dev = [torch.from_numpy(getattr(w, k)).to(device).reshape(-1) for k in w.HOST_FIELDS]
-    return nbos_snapshot_create(w.n_snapshots, w.n_hosts, torch.from_numpy(w.limit_num),
-                                torch.from_numpy(w.limit_den), *dev, replicas_R=w.replicas_R,
+    own = bool(flags & NBOS_LIMIT_CLUSTER_SR)
+    return nbos_snapshot_create(w.n_snapshots, w.n_hosts, None if own else torch.from_numpy(w.limit_num),
+                                None if own else torch.from_numpy(w.limit_den), *dev, replicas_R=w.replicas_R,
                                 key_order=key_order, flags=flags, stream=stream)
 
 

@@ -41,7 +41,7 @@ int check_desc_scalars(const nbos_snapshot_desc *d)
         return fail(NBOS_ERR_INVALID_ARG, "n_snapshots must be in 1..65535 (got %d)", d->n_snapshots);
     if (d->n_hosts < 1 || d->n_hosts > NBOS_MAX_HOSTS)
         return fail(NBOS_ERR_INVALID_ARG, "n_hosts must be in 1..%d (got %d)", NBOS_MAX_HOSTS, d->n_hosts);
-    if (d->flags & ~(NBOS_REQUIRE_IDLE_GPUS | NBOS_FORCE_KEY64))
+    if (d->flags & ~(NBOS_REQUIRE_IDLE_GPUS | NBOS_FORCE_KEY64 | NBOS_LIMIT_CLUSTER_SR))
         return fail(NBOS_ERR_INVALID_ARG, "unknown bits in flags (0x%x)", d->flags);
     return NBOS_OK;
 }
@@ -55,12 +55,13 @@ int check_desc_full(const nbos_snapshot_desc *d)
     if (d->key_order != NBOS_KEY_IDLE_FIRST && d->key_order != NBOS_KEY_SR_FIRST)
         return fail(NBOS_ERR_INVALID_ARG, "unknown key_order %d", d->key_order);
     if (d->reserved != 0) return fail(NBOS_ERR_INVALID_ARG, "reserved must be 0");
-    if (!d->limit_num || !d->limit_den) return fail(NBOS_ERR_INVALID_ARG, "limit_num / limit_den is NULL");
+    const bool own_limit = (d->flags & NBOS_LIMIT_CLUSTER_SR) != 0;
+    if (!own_limit && (!d->limit_num || !d->limit_den)) return fail(NBOS_ERR_INVALID_ARG, "limit_num / limit_den is NULL");
     const void *arrays[6] = {d->gpus_total, d->gpus_subscribed, d->gpus_committed,
                              d->vram_gb, d->millicpus, d->mem_mb};
     for (int i = 0; i < 6; ++i)
         if (!arrays[i]) return fail(NBOS_ERR_INVALID_ARG, "host-state array %d is NULL", i);
-    for (int n = 0; n < d->n_snapshots; ++n) {
+    for (int n = 0; n < d->n_snapshots && !own_limit; ++n) {
         if (d->limit_den[n] < 1) return fail(NBOS_ERR_INVALID_ARG, "limit_den[%d] must be >= 1", n);
         if (d->limit_num[n] < 0) return fail(NBOS_ERR_INVALID_ARG, "limit_num[%d] must be >= 0", n);
     }

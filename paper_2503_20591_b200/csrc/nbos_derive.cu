@@ -17,20 +17,71 @@ namespace {
 
 struct ScanArgs {
     const int32_t *G, *S, *C, *AV, *AC, *AM;
-    const int2 *limits;  // per snapshot (num, den)
+    const longlong2 *limits;  // per snapshot (num * R, den): cap = floor(limits.x * G / limits.y)
     SnapStats *stats;
     int H, R, flags;
 };
 
-__device__ __forceinline__ int derive_gmax(long long G, long long S, long long C, long long num,
-                                           long long den, long long R, int flags)
+// `num_r` is the limit's numerator times R (R already cancelled for the dynamic limit).
+__device__ __forceinline__ int derive_gmax(long long G, long long S, long long C, long long num_r,
+                                           long long den, int flags)
 {
-    if (G < 1) return -1;
-    long long cap = (num * G * R) / den;
+    if (G < 1 || den < 1) return -1;
+    long long cap = (num_r * G) / den;
     long long gm = cap - S;
     if (gm > G) gm = G;
     if ((flags & NBOS_REQUIRE_IDLE_GPUS) && gm > G - C) gm = G - C;
     return gm < 0 ? -1 : (int)gm;
+}
+
+// Cluster sums of Sections 3.4.1 / 3.4.2: sums[n] = (sum G, sum S, sum C, unused) per snapshot.
+// grid (blocks_per_snapshot, N); `sums` must be zeroed before the launch.
+__global__ void __launch_bounds__(256) sums_kernel(const int32_t *G, const int32_t *S, const int32_t *C,
+                                                   int H, unsigned long long *sums)
+{
+    __shared__ unsigned long long s_sum[3];
+    if (threadIdx.x < 3) s_sum[threadIdx.x] = 0ull;
+    __syncthreads();
+    const int n = blockIdx.y;
+    unsigned long long g = 0, s = 0, c = 0;
+    for (int h = blockIdx.x * blockDim.x + threadIdx.x; h < H; h += gridDim.x * blockDim.x) {
+        const size_t i = (size_t)n * H + h;
+        g += (unsigned long long)(long long)G[i];
+        s += (unsigned long long)(long long)S[i];
+        c += (unsigned long long)(long long)C[i];
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        g += __shfl_xor_sync(0xFFFFFFFFu, g, off);
+        s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
+        c += __shfl_xor_sync(0xFFFFFFFFu, c, off);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        atomicAdd(&s_sum[0], g);
+        atomicAdd(&s_sum[1], s);
+        atomicAdd(&s_sum[2], c);
+    }
+    __syncthreads();
+    if (threadIdx.x < 3) atomicAdd(&sums[(size_t)n * 4 + threadIdx.x], s_sum[threadIdx.x]);
+}
+
+// Dynamic cluster-wide limit (Section 3.4.1, third factor): sum S / (sum G * R). R cancels against
+// the R of the per-host ratio, so the stored pair is (sum S, sum G).
+__global__ void limits_from_sums_kernel(const unsigned long long *sums, longlong2 *limits, int N)
+{
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n < N) limits[n] = make_longlong2((long long)sums[(size_t)n * 4 + 1], (long long)sums[(size_t)n * 4 + 0]);
+}
+
+// Auto-scaler rule (Section 3.4.2) next to the sums: sums[n*4+3] = +1 if sum G < f * sum C (scale
+// out), -1 if f * sum C < sum G (servers may be released), 0 if equal; f = f_num / f_den.
+__global__ void autoscale_kernel(unsigned long long *sums, int N, long long f_num, long long f_den)
+{
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= N) return;
+    const long long have = f_den * (long long)sums[(size_t)n * 4 + 0];
+    const long long expected = f_num * (long long)sums[(size_t)n * 4 + 2];
+    sums[(size_t)n * 4 + 3] = (unsigned long long)(long long)((have < expected) - (expected < have));
 }
 
 // grid (blocks_per_snapshot, N). Validates the value ranges and reduces what the key layout
@@ -52,7 +103,7 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
         s_sub_max = 0ull;
     }
     __syncthreads();
-    const int2 lim = a.limits[n];
+    const longlong2 lim = a.limits[n];
     unsigned int err = 0u;
     int idle_max = 0, g_min_inv = 0;  // INT_MAX - smallest G seen, 0 = none
     unsigned long long sub_max = 0ull;
@@ -69,7 +120,7 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
             g_min_inv = max(g_min_inv, INT_MAX - G);
         }
         idle_max = max(idle_max, G - C);
-        const int gm = derive_gmax(G, S, C, lim.x, lim.y, a.R, a.flags);
+        const int gm = derive_gmax(G, S, C, lim.x, lim.y, a.flags);
         if (gm >= 0) sub_max = max(sub_max, (unsigned long long)S + (unsigned long long)gm);
         max_gcap1 = max(max_gcap1, gm + 1);
         max_av = max(max_av, a.AV[i]);
@@ -101,7 +152,7 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
 
 struct EmitArgs {
     const int32_t *G, *S, *C, *AV, *AC, *AM;
-    const int2 *limits;
+    const longlong2 *limits;
     const long long *lambda;  // per snapshot
     int4 *feas;                 // records in host-index order (staging)
     void *ab;
@@ -127,8 +178,8 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
     if (h < a.H) {
         const size_t i = (size_t)n * a.H + h;
         const int G = a.G[i], S = a.S[i], C = a.C[i];
-        const int2 lim = a.limits[n];
-        const int gm = derive_gmax(G, S, C, lim.x, lim.y, a.R, a.flags);
+        const longlong2 lim = a.limits[n];
+        const int gm = derive_gmax(G, S, C, lim.x, lim.y, a.flags);
         f = make_int4(gm, a.AV[i], a.AC[i], a.AM[i]);
         if (gm >= 0) {
             const KeyT w = (KeyT)(a.lambda[n] / G);
@@ -236,7 +287,8 @@ Layout workspace_layout(int N, int Hpad)
     Layout l;
     size_t o = 0;
     l.off_status = o;  o = up(o + 256);
-    l.off_limits = o;  o = up(o + (size_t)N * sizeof(int2));
+    l.off_limits = o;  o = up(o + (size_t)N * sizeof(longlong2));
+    l.off_sums = o;    o = up(o + (size_t)N * 4 * sizeof(unsigned long long));
     l.off_lambda = o;  o = up(o + (size_t)N * sizeof(long long));
     l.off_stats = o;   o = up(o + (size_t)N * sizeof(SnapStats));
     l.off_feas = o;    o = up(o + (size_t)N * Hpad * sizeof(int4));
@@ -250,6 +302,19 @@ Layout workspace_layout(int N, int Hpad)
     return l;
 }
 
+int launch_cluster_sums(const int32_t *d_G, const int32_t *d_S, const int32_t *d_C, int N, int H,
+                        long long f_num, long long f_den, long long *d_out, cudaStream_t stream)
+{
+    unsigned long long *sums = reinterpret_cast<unsigned long long *>(d_out);
+    NBOS_CUDA_TRY(cudaMemsetAsync(sums, 0, sizeof(unsigned long long) * 4 * (size_t)N, stream));
+    int bx = (H + 255) / 256;
+    if (bx > 64) bx = 64;
+    sums_kernel<<<dim3(bx, N), 256, 0, stream>>>(d_G, d_S, d_C, H, sums);
+    autoscale_kernel<<<(N + 255) / 256, 256, 0, stream>>>(sums, N, f_num, f_den);
+    NBOS_CUDA_TRY(cudaGetLastError());
+    return NBOS_OK;
+}
+
 int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t *d_G,
                     const int32_t *d_S, const int32_t *d_C, const int32_t *d_AV,
                     const int32_t *d_AC, const int32_t *d_AM, cudaStream_t stream)
@@ -257,12 +322,14 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     const int N = s->N, H = s->H, Hpad = s->Hpad;
     const Layout lay = workspace_layout(N, Hpad);
     char *ws = static_cast<char *>(s->workspace);
-    int2 *d_limits = reinterpret_cast<int2 *>(ws + lay.off_limits);
+    longlong2 *d_limits = reinterpret_cast<longlong2 *>(ws + lay.off_limits);
+    unsigned long long *d_sums = reinterpret_cast<unsigned long long *>(ws + lay.off_sums);
+    const bool dynamic_limit = (s->flags & NBOS_LIMIT_CLUSTER_SR) != 0;
     long long *d_lambda = reinterpret_cast<long long *>(ws + lay.off_lambda);
     SnapStats *d_stats = reinterpret_cast<SnapStats *>(ws + lay.off_stats);
 
     // limits -> device
-    int2 *h_limits = static_cast<int2 *>(malloc(sizeof(int2) * (size_t)N));
+    longlong2 *h_limits = static_cast<longlong2 *>(malloc(sizeof(longlong2) * (size_t)N));
     SnapStats *h_stats = static_cast<SnapStats *>(malloc(sizeof(SnapStats) * (size_t)N));
     long long *h_lambda = static_cast<long long *>(malloc(sizeof(long long) * (size_t)N));
     struct Free {
@@ -270,16 +337,23 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
         ~Free() { free(a); free(b); free(c); }
     } guard{h_limits, h_stats, h_lambda};
     if (!h_limits || !h_stats || !h_lambda) return fail(NBOS_ERR_NO_MEMORY, "host allocation failed");
-    for (int n = 0; n < N; ++n) h_limits[n] = make_int2(d->limit_num[n], d->limit_den[n]);
+    if (!dynamic_limit)
+        for (int n = 0; n < N; ++n) h_limits[n] = make_longlong2((long long)d->limit_num[n] * s->R, d->limit_den[n]);
 
     // status word, limits, lambda and scan statistics are contiguous: one clear
     NBOS_CUDA_TRY(cudaMemsetAsync(ws + lay.off_status, 0, lay.off_feas - lay.off_status, stream));
-    NBOS_CUDA_TRY(cudaMemcpyAsync(d_limits, h_limits, sizeof(int2) * (size_t)N,
-                                  cudaMemcpyHostToDevice, stream));
-
-    ScanArgs sa{d_G, d_S, d_C, d_AV, d_AC, d_AM, d_limits, d_stats, H, s->R, s->flags};
     int bx = (H + 255) / 256;
     if (bx > 64) bx = 64;
+    if (dynamic_limit) {
+        sums_kernel<<<dim3(bx, N), 256, 0, stream>>>(d_G, d_S, d_C, H, d_sums);
+        limits_from_sums_kernel<<<(N + 255) / 256, 256, 0, stream>>>(d_sums, d_limits, N);
+        NBOS_CUDA_TRY(cudaGetLastError());
+    } else {
+        NBOS_CUDA_TRY(cudaMemcpyAsync(d_limits, h_limits, sizeof(longlong2) * (size_t)N,
+                                      cudaMemcpyHostToDevice, stream));
+    }
+
+    ScanArgs sa{d_G, d_S, d_C, d_AV, d_AC, d_AM, d_limits, d_stats, H, s->R, s->flags};
     scan_kernel<<<dim3(bx, N), 256, 0, stream>>>(sa);
     NBOS_CUDA_TRY(cudaGetLastError());
     NBOS_CUDA_TRY(cudaMemcpyAsync(h_stats, d_stats, sizeof(SnapStats) * (size_t)N,

@@ -37,7 +37,7 @@ enum : unsigned int {
 };
 
 struct Layout {
-    size_t off_status, off_limits, off_lambda, off_stats, off_feas, off_ab, off_pk;
+    size_t off_status, off_limits, off_sums, off_lambda, off_stats, off_feas, off_ab, off_pk;
     size_t off_tmp_feas, off_tmp_ab, off_sortkey, off_perm, total;
 };
 Layout workspace_layout(int n_snapshots, int hosts_padded);
@@ -88,6 +88,10 @@ namespace nbos {
 int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *host_desc, const int32_t *d_G,
                     const int32_t *d_S, const int32_t *d_C, const int32_t *d_AV,
                     const int32_t *d_AC, const int32_t *d_AM, cudaStream_t stream);
+
+// Cluster sums + auto-scaler sign per snapshot into d_out [N][4] (nbos_derive.cu).
+int launch_cluster_sums(const int32_t *d_G, const int32_t *d_S, const int32_t *d_C, int N, int H,
+                        long long f_num, long long f_den, long long *d_out, cudaStream_t stream);
 
 // a1-a9: the placement launch (nbos_place.cu). The pointers are those of the whole batch; the
 // launch handles the flattened requests [range_first, range_first + range_count) of the N * batch
