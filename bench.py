@@ -376,8 +376,24 @@ def run_ours(args):
             torch.cuda.synchronize()
             ms = a.elapsed_time(b) / reps
             info = sn.info()
+            # first-fit variant (stops at the third feasible host): decisions/s only
+            ff = nb.launch_config(first_fit=1)
+            oh2 = torch.empty_like(oh)
+            for _ in range(3):
+                nb.nbos_place_batch(sn, rq, oh2, of, stream=stream, config=ff)
+            torch.cuda.synchronize()
+            a.record(stream)
+            for _ in range(reps):
+                nb.nbos_place_batch(sn, rq, oh2, of, stream=stream, config=ff)
+            b.record(stream)
+            torch.cuda.synchronize()
+            ms_ff = a.elapsed_time(b) / reps
             others[ww.name] = {"kernel_ms": ms, "decisions_per_s": ww.decisions / ms * 1e3,
                                "pairs_per_s": ww.pairs / ms * 1e3,
+                               "first_fit_kernel_ms": ms_ff,
+                               "first_fit_decisions_per_s": ww.decisions / ms_ff * 1e3,
+                               "first_fit_stream_gbs": ww.decisions * 32 / (ms_ff * 1e-3) / 1e9,
+                               "first_fit_same_output": bool(torch.equal(oh, oh2)),
                                "found_histogram": torch.bincount(of.flatten(), minlength=4).tolist(),
                                "packed_test": info.packed_test, "static_key": info.static_key,
                                "note": "same inputs every launch (L2-resident), back-to-back launches"}

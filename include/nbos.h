@@ -131,6 +131,12 @@ typedef struct nbos_snapshot_info {
  *                      0 = the fastest form the snapshot allows; 1 = four separate capacity
  *                      compares; 2 = packed capacity test with the key computed per pair (even if
  *                      the snapshot would allow ranking by the host part of the key alone).
+ *   first_fit          1 = stop scanning a request's hosts at the third feasible one. Possible
+ *                      when every host has the same key slope and the table is stored in key
+ *                      order (nbos_snapshot_info: static_key and presorted), because then the
+ *                      first three feasible hosts in table order are the best three; otherwise
+ *                      the flag is ignored. Same outputs, far fewer (request, host) pairs looked
+ *                      at: throughput of this variant is not a pairs/s figure.
  */
 typedef struct nbos_launch_config {
     int32_t lanes_per_request;
@@ -139,7 +145,8 @@ typedef struct nbos_launch_config {
     int32_t tile_hosts;
     int32_t grid_blocks;
     int32_t pair_mode;
-    int32_t reserved[2]; /* must be 0 */
+    int32_t first_fit;
+    int32_t reserved; /* must be 0 */
 } nbos_launch_config;
 
 /* Device bytes nbos_snapshot_create needs in `workspace` for this N and H (Section 3.4.1 state

@@ -84,7 +84,7 @@ class nbos_launch_config(ctypes.Structure):
         ("lanes_per_request", ctypes.c_int32), ("requests_per_lane", ctypes.c_int32),
         ("host_split", ctypes.c_int32), ("tile_hosts", ctypes.c_int32),
         ("grid_blocks", ctypes.c_int32), ("pair_mode", ctypes.c_int32),
-        ("reserved", ctypes.c_int32 * 2),
+        ("first_fit", ctypes.c_int32), ("reserved", ctypes.c_int32),
     ]
 
 
@@ -398,11 +398,12 @@ def nbos_probe_wait_timeout(limit_ns: int, stream=None):
 
 
 def launch_config(lanes_per_request=0, requests_per_lane=0, host_split=0, tile_hosts=0,
-                  grid_blocks=0, pair_mode=0) -> nbos_launch_config:
+                  grid_blocks=0, pair_mode=0, first_fit=0) -> nbos_launch_config:
     c = nbos_launch_config()
     c.lanes_per_request, c.requests_per_lane = lanes_per_request, requests_per_lane
     c.host_split, c.tile_hosts, c.grid_blocks = host_split, tile_hosts, grid_blocks
     c.pair_mode = pair_mode
+    c.first_fit = first_fit
     return c
 
 

@@ -185,6 +185,29 @@ def test_packed_test_layouts_and_fallback(nb):
     assert_same(got, ref, "asks at the capacity maxima")
 
 
+def test_first_fit_variant(nb):
+    """Stopping at the third feasible host (table in key order, same key slope everywhere) gives
+    the same bytes as the full evaluation; where the conditions do not hold the flag is ignored."""
+    cfg = nb.launch_config(first_fit=1)
+    for w in (W.make_config(0), W.make_config(1), W.make_config(2, batch=40_000),
+              W.make_config(3, batch=20_000), W.make_config(4, batch=300, n_snapshots=64),
+              W.uniform_cluster(9000, 500, seed=5), W.uniform_cluster(33, 7, seed=6),
+              W.mixed_gpu_cluster(700, 3000, seed=7),          # not static: flag ignored
+              W.uniform_cluster(70000, 40, seed=8)):           # not presorted: flag ignored
+        for key_order in (0, 1):
+            for lib_flags in (0, 2):
+                got, ref = both(nb, w, key_order=key_order, config=cfg, lib_flags=lib_flags)
+                assert_same(got, ref, f"first fit {w.name} order={key_order} lib={lib_flags}")
+    w = W.make_config(2, batch=10_000)
+    got, ref = both(nb, w, flags=1, config=cfg)
+    assert_same(got, ref, "first fit, idle reading")
+    w = W.make_config(1, batch=2000)
+    w.mem_mb[0, 9] = (1 << 31) - 1                              # no packed table: plain compares
+    w.requests[0, :50, 0] = -3
+    got, ref = both(nb, w, config=cfg)
+    assert_same(got, ref, "first fit, plain table")
+
+
 def test_large_tables(nb):
     """Up to 65,536 hosts the table is stored in key order; beyond that it stays in host order.
     Results are the same either way."""
