@@ -70,6 +70,9 @@ extern "C" {
                                   * sum(S) / (sum(G) * R), as its limit. An empty cluster (sum S = 0)
                                   * then admits only g = 0; the paper gives no floor.          */
 
+#define NBOS_ROOM_FOR_COMMITS 8   /* size the key's ratio field for subscribed counts growing up to each
+                                  * host's cap; required by nbos_place_batch_sequential          */
+
 #define NBOS_MAX_HOSTS (1 << 20)   /* per snapshot                          */
 #define NBOS_MAX_GPUS_PER_HOST 1023
 #define NBOS_MAX_REPLICAS 1024
@@ -93,7 +96,8 @@ typedef struct nbos_snapshot_desc {
     int32_t n_hosts;     /* 1 <= H <= NBOS_MAX_HOSTS                  */
     int32_t replicas_R;  /* 1 .. NBOS_MAX_REPLICAS; the paper uses 3  */
     int32_t key_order;   /* NBOS_KEY_*                                */
-    int32_t flags;       /* NBOS_REQUIRE_IDLE_GPUS | NBOS_FORCE_KEY64 | NBOS_LIMIT_CLUSTER_SR */
+    int32_t flags;       /* NBOS_REQUIRE_IDLE_GPUS | NBOS_FORCE_KEY64 | NBOS_LIMIT_CLUSTER_SR |
+                          * NBOS_ROOM_FOR_COMMITS */
     int32_t reserved;    /* must be 0                                 */
     const int32_t *limit_num; /* HOST [N] in both create variants     */
     const int32_t *limit_den; /* HOST [N]                             */
@@ -284,6 +288,27 @@ typedef struct nbos_cluster_state {
 int nbos_select_executors(const nbos_cluster_state *state, const int32_t *requests,
                           const int32_t *replica_hosts, int64_t n_kernels, int32_t *out_executor,
                           int32_t *out_can_run, void *cuda_stream);
+
+/*
+ * Sequential placement with commits: the paper's scheduler places one kernel at a time, and a
+ * placed kernel's replicas subscribe its GPUs on their three servers before the next kernel is
+ * looked at (Sections 3.2.1, 3.4.1). For request i = 0, 1, ... of each snapshot, in order: the
+ * same decision as nbos_place_batch against the current state; if three hosts were found, S of
+ * each grows by the request's GPU count (its key and its remaining room under the SR limit move
+ * accordingly); if fewer were found nothing changes (the kernel is not created). Committed GPUs
+ * and the other capacities stay as they are. Snapshots are independent and run in parallel; the
+ * snapshot object itself is not modified.
+ *   snap            must have been created with NBOS_ROOM_FOR_COMMITS; at most
+ *                   NBOS_SEQUENTIAL_MAX_HOSTS hosts (the evolving state lives on one SM);
+ *                   otherwise INVALID_ARG / RANGE
+ *   requests, out_hosts, out_found   as for nbos_place_batch
+ *   out_subscribed  DEVICE [N * H] int32 or NULL: S of every host after the last request
+ * Asynchronous on `cuda_stream`.
+ */
+#define NBOS_SEQUENTIAL_MAX_HOSTS 8192
+int nbos_place_batch_sequential(const nbos_snapshot *snap, const int32_t *requests,
+                                int64_t batch_per_snapshot, int32_t *out_hosts, int32_t *out_found,
+                                int32_t *out_subscribed, void *cuda_stream);
 
 /*
  * Cluster sums and the auto-scaler rule (Sections 3.4.1, 3.4.2), per snapshot:

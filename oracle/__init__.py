@@ -14,6 +14,7 @@ from .placement import (  # noqa: F401
     compare_sr_after,
     feasible,
     place,
+    place_sequential,
     place_workload,
     ranks_before,
     scale_out_deficit,

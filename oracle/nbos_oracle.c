@@ -267,3 +267,40 @@ void nbos_oracle_scale_out_deficit(const int32_t *found, int64_t batch, int64_t 
         }
     }
 }
+
+/*
+ * Sequential placement: the paper's scheduler places one kernel at a time, and the replicas of a
+ * placed kernel subscribe to its GPUs on their three servers before the next kernel is looked at
+ * (Section 3.2.1: "the kernel replicas subscribe to the requested resources"; Section 3.4.1: S is
+ * the sum of the GPUs requested by all replicas scheduled on the server).
+ *
+ * For request r = 0, 1, ... in order: place it against the current state exactly as
+ * nbos_oracle_place does; if three servers were found, add g to S on each of them; if fewer were
+ * found the kernel is not created (the scheduler scales out and retries later, Section 3.2.1) and
+ * nothing changes. Committed GPUs C and the other capacities are not touched: a new replica is
+ * idle until a cell runs.
+ *   S_final [n_hosts] receives the subscribed GPUs after the last request (may be NULL).
+ */
+int nbos_oracle_place_sequential(const nbos_oracle_cluster *cl, const int32_t *requests,
+                                 int64_t batch, int32_t *out_hosts, int32_t *out_found,
+                                 int32_t *S_final)
+{
+    if (!cl || cl->n_hosts < 0 || batch < 0) return -1;
+    int32_t *S_now = (int32_t *)malloc(sizeof(int32_t) * (size_t)(cl->n_hosts > 0 ? cl->n_hosts : 1));
+    if (!S_now) return -1;
+    for (int32_t h = 0; h < cl->n_hosts; ++h) S_now[h] = cl->S[h];
+    nbos_oracle_cluster now = *cl;
+    now.S = S_now;
+    int rc = 0;
+    for (int64_t r = 0; r < batch && rc == 0; ++r) {
+        int32_t found = 0;
+        rc = nbos_oracle_place(&now, requests + 4 * r, 1, out_hosts + 3 * r, &found);
+        if (out_found) out_found[r] = found;
+        if (rc == 0 && found == NBOS_ORACLE_REPLICAS_PLACED)
+            for (int k = 0; k < NBOS_ORACLE_REPLICAS_PLACED; ++k) S_now[out_hosts[3 * r + k]] += requests[4 * r];
+    }
+    if (S_final)
+        for (int32_t h = 0; h < cl->n_hosts; ++h) S_final[h] = S_now[h];
+    free(S_now);
+    return rc;
+}

@@ -68,6 +68,9 @@ def _load():
         lib.nbos_oracle_select_executors.restype = ctypes.c_int
         lib.nbos_oracle_select_executors.argtypes = [ctypes.POINTER(_Cluster), _i32p, _i32p,
                                                      ctypes.c_int64, _i32p, _i32p]
+        lib.nbos_oracle_place_sequential.restype = ctypes.c_int
+        lib.nbos_oracle_place_sequential.argtypes = [ctypes.POINTER(_Cluster), _i32p, ctypes.c_int64,
+                                                     _i32p, _i32p, _i32p]
         i64p = ctypes.POINTER(ctypes.c_int64)
         lib.nbos_oracle_cluster_sums.restype = None
         lib.nbos_oracle_cluster_sums.argtypes = [ctypes.POINTER(_Cluster), i64p]
@@ -147,6 +150,25 @@ def select_executors(G, S, C, AV, AC, AM, requests, replica_hosts, replicas_R=3)
     if rc != 0:
         raise ValueError("nbos_oracle_select_executors rejected its arguments")
     return ex, mask
+
+
+def place_sequential(G, S, C, AV, AC, AM, limit_num, limit_den, requests, replicas_R=3,
+                     key_order=KEY_IDLE_FIRST, flags=0):
+    """One snapshot, requests placed one after the other; a request that finds three hosts adds
+    its GPUs to their subscribed count before the next one is placed.
+    Returns (hosts [B,3], found [B], S_final [H])."""
+    cl, keep = _cluster(G, S, C, AV, AC, AM, limit_num, limit_den, replicas_R, key_order, flags)
+    req = _as_i32(requests).reshape(-1, 4)
+    b = req.shape[0]
+    hosts = np.empty((b, 3), dtype=np.int32)
+    found = np.empty((b,), dtype=np.int32)
+    s_final = np.empty((cl.n_hosts,), dtype=np.int32)
+    rc = _load().nbos_oracle_place_sequential(ctypes.byref(cl), req.ctypes.data_as(_i32p), b,
+                                              hosts.ctypes.data_as(_i32p), found.ctypes.data_as(_i32p),
+                                              s_final.ctypes.data_as(_i32p))
+    if rc != 0:
+        raise ValueError("nbos_oracle_place_sequential rejected its arguments")
+    return hosts, found, s_final
 
 
 def cluster_sums(G, S, C, replicas_R=3):

@@ -28,6 +28,7 @@ NBOS_KEY_SR_FIRST = 1
 NBOS_REQUIRE_IDLE_GPUS = 1
 NBOS_FORCE_KEY64 = 2
 NBOS_LIMIT_CLUSTER_SR = 4
+NBOS_ROOM_FOR_COMMITS = 8
 
 NBOS_PROBE_MIX_ALU = 0
 NBOS_PROBE_MIX_IMAD = 1
@@ -38,7 +39,7 @@ EXPORTED_SYMBOLS = (
     "nbos_snapshot_workspace_bytes", "nbos_snapshot_create", "nbos_snapshot_create_host",
     "nbos_snapshot_destroy", "nbos_snapshot_get_info", "nbos_place_batch", "nbos_place_batch_ex",
     "nbos_place_batch_host", "nbos_place_batch_noalloc", "nbos_select_executors",
-    "nbos_cluster_sums", "nbos_scale_out_deficit",
+    "nbos_cluster_sums", "nbos_scale_out_deficit", "nbos_place_batch_sequential",
     "nbos_snapshot_status", "nbos_strerror", "nbos_last_error_detail",
     "nbos_probe_int32_issue", "nbos_probe_wait_timeout",
 )
@@ -121,6 +122,7 @@ def load_library() -> ctypes.CDLL:
     lib.nbos_select_executors.argtypes = [P(nbos_cluster_state), vp, vp, i64, vp, vp, vp]
     lib.nbos_cluster_sums.argtypes = [vp, vp, vp] + [ctypes.c_int32] * 4 + [vp, vp]
     lib.nbos_scale_out_deficit.argtypes = [vp, ctypes.c_int32, i64, vp, vp]
+    lib.nbos_place_batch_sequential.argtypes = [vp, vp, i64, vp, vp, vp, vp]
     lib.nbos_snapshot_status.argtypes = [vp, vp]
     lib.nbos_strerror.argtypes = [ctypes.c_int]
     lib.nbos_strerror.restype = ctypes.c_char_p
@@ -379,6 +381,27 @@ def nbos_scale_out_deficit(found, n_snapshots, out_deficit, stream=None) -> None
         raise ValueError("out_deficit must be a CUDA int64 tensor of n_snapshots * 2 elements")
     _check(load_library().nbos_scale_out_deficit(_ptr(found), n_snapshots, found.numel() // n_snapshots,
                                                  _ptr(out_deficit), _stream_ptr(stream)))
+
+
+def nbos_place_batch_sequential(snap: Snapshot, requests, out_hosts, out_found=None,
+                                out_subscribed=None, stream=None) -> None:
+    """Device tensors as for nbos_place_batch, plus out_subscribed [N,H] int32 or None. The
+    snapshot must have been created with NBOS_ROOM_FOR_COMMITS."""
+    lib = load_library()
+    _i32(requests, "requests", "cuda")
+    _i32(out_hosts, "out_hosts", "cuda")
+    for n, t in (("out_found", out_found), ("out_subscribed", out_subscribed)):
+        if t is not None:
+            _i32(t, n, "cuda")
+    b = _batch_of(snap, requests)
+    if out_hosts.numel() != snap.n_snapshots * b * 3:
+        raise ValueError("out_hosts must hold n_snapshots * batch * 3 values")
+    if out_found is not None and out_found.numel() != snap.n_snapshots * b:
+        raise ValueError("out_found must hold n_snapshots * batch values")
+    if out_subscribed is not None and out_subscribed.numel() != snap.n_snapshots * snap.n_hosts:
+        raise ValueError("out_subscribed must hold n_snapshots * n_hosts values")
+    _check(lib.nbos_place_batch_sequential(snap.handle, _ptr(requests), b, _ptr(out_hosts),
+                                           _ptr(out_found), _ptr(out_subscribed), _stream_ptr(stream)))
 
 
 def nbos_probe_int32_issue(mix: int, iters: int, blocks: int, threads: int, stream=None):

@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libnbos.so")
-SOURCES = ("nbos_api.cu", "nbos_derive.cu", "nbos_place.cu", "nbos_executor.cu", "nbos_cluster.cu", "nbos_probe.cu")
+SOURCES = ("nbos_api.cu", "nbos_derive.cu", "nbos_place.cu", "nbos_executor.cu", "nbos_cluster.cu", "nbos_sequential.cu", "nbos_probe.cu")
 HEADERS = (os.path.join(ROOT, "include", "nbos.h"), os.path.join(ROOT, "include", "nbos_probe.h"),
            os.path.join(CSRC, "nbos_internal.h"))
 ARCH_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a"]

@@ -41,7 +41,7 @@ int check_desc_scalars(const nbos_snapshot_desc *d)
         return fail(NBOS_ERR_INVALID_ARG, "n_snapshots must be in 1..65535 (got %d)", d->n_snapshots);
     if (d->n_hosts < 1 || d->n_hosts > NBOS_MAX_HOSTS)
         return fail(NBOS_ERR_INVALID_ARG, "n_hosts must be in 1..%d (got %d)", NBOS_MAX_HOSTS, d->n_hosts);
-    if (d->flags & ~(NBOS_REQUIRE_IDLE_GPUS | NBOS_FORCE_KEY64 | NBOS_LIMIT_CLUSTER_SR))
+    if (d->flags & ~(NBOS_REQUIRE_IDLE_GPUS | NBOS_FORCE_KEY64 | NBOS_LIMIT_CLUSTER_SR | NBOS_ROOM_FOR_COMMITS))
         return fail(NBOS_ERR_INVALID_ARG, "unknown bits in flags (0x%x)", d->flags);
     return NBOS_OK;
 }
@@ -364,6 +364,24 @@ int nbos_place_batch_noalloc(const nbos_snapshot *snap, const int32_t *requests,
     if (!aligned(out_hosts, 4) || !aligned(out_found, 4)) return fail(NBOS_ERR_INVALID_ARG, "output not 4-byte aligned");
     return launch_place_static(snap, requests, batch_per_snapshot, out_hosts, out_found,
                                static_cast<cudaStream_t>(cuda_stream), host_split);
+}
+
+int nbos_place_batch_sequential(const nbos_snapshot *snap, const int32_t *requests,
+                                int64_t batch_per_snapshot, int32_t *out_hosts, int32_t *out_found,
+                                int32_t *out_subscribed, void *cuda_stream)
+{
+    if (!snap) return fail(NBOS_ERR_INVALID_ARG, "snapshot is NULL");
+    if (!(snap->flags & NBOS_ROOM_FOR_COMMITS))
+        return fail(NBOS_ERR_INVALID_ARG, "the snapshot was not created with NBOS_ROOM_FOR_COMMITS");
+    if (snap->Hpad > NBOS_SEQUENTIAL_MAX_HOSTS)
+        return fail(NBOS_ERR_RANGE, "sequential placement supports at most %d hosts (snapshot has %d)",
+                    NBOS_SEQUENTIAL_MAX_HOSTS, snap->H);
+    if (batch_per_snapshot < 0 || batch_per_snapshot > ((int64_t)1 << 40) / snap->N)
+        return fail(NBOS_ERR_INVALID_ARG, "batch_per_snapshot out of range");
+    if (batch_per_snapshot != 0 && (!requests || !out_hosts)) return fail(NBOS_ERR_INVALID_ARG, "requests / out_hosts is NULL");
+    if (!aligned(requests, 16)) return fail(NBOS_ERR_INVALID_ARG, "requests is not 16-byte aligned");
+    return launch_place_sequential(snap, requests, batch_per_snapshot, out_hosts, out_found, out_subscribed,
+                                   static_cast<cudaStream_t>(cuda_stream));
 }
 
 int nbos_snapshot_status(const nbos_snapshot *snap, void *cuda_stream)

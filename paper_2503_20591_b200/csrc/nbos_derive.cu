@@ -121,7 +121,13 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
         }
         idle_max = max(idle_max, G - C);
         const int gm = derive_gmax(G, S, C, lim.x, lim.y, a.flags);
-        if (gm >= 0) sub_max = max(sub_max, (unsigned long long)S + (unsigned long long)gm);
+        if (gm >= 0) {
+            // largest S + g the ratio field has to hold: what fits now, or -- when later commits may
+            // add to S (NBOS_ROOM_FOR_COMMITS) -- everything up to the host's cap
+            unsigned long long top = (unsigned long long)S + (unsigned long long)gm;
+            if (a.flags & NBOS_ROOM_FOR_COMMITS) top = max(top, (unsigned long long)((lim.x * (long long)G) / lim.y));
+            sub_max = max(sub_max, top);
+        }
         max_gcap1 = max(max_gcap1, gm + 1);
         max_av = max(max_av, a.AV[i]);
         max_ac = max(max_ac, a.AC[i]);
@@ -155,6 +161,7 @@ struct EmitArgs {
     const longlong2 *limits;
     const long long *lambda;  // per snapshot
     int4 *feas;                 // records in host-index order (staging)
+    int4 *seq;                  // (min(G, idle), cap - S, S, 0) per host, for sequential placement
     void *ab;
     unsigned long long *sortkey;  // [N][Hpad] visiting-order key: A, or near-max for hosts that take nothing
     int H, Hpad, R, flags, key_order;
@@ -173,6 +180,7 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
     const int h = blockIdx.x * blockDim.x + threadIdx.x;
     if (h >= a.Hpad) return;
     int4 f = make_int4(-1, 0, 0, 0);  // padding host: takes nothing
+    int4 sq = make_int4(-1, -1, 0, 0);
     KeyT A = (KeyT)h, B = 0;
     unsigned long long sk = kSortNever | (unsigned int)h;
     if (h < a.H) {
@@ -181,6 +189,13 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
         const longlong2 lim = a.limits[n];
         const int gm = derive_gmax(G, S, C, lim.x, lim.y, a.flags);
         f = make_int4(gm, a.AV[i], a.AC[i], a.AM[i]);
+        sq.z = S;
+        if (G >= 1 && lim.y >= 1) {
+            long long room = (lim.x * (long long)G) / lim.y - S;   // cap - S
+            room = room > INT_MAX ? INT_MAX : room < -1 ? -1 : room;
+            const int g_cap = (a.flags & NBOS_REQUIRE_IDLE_GPUS) ? min(G, G - C) : G;
+            sq = make_int4(g_cap, (int)room, S, 0);
+        }
         if (gm >= 0) {
             const KeyT w = (KeyT)(a.lambda[n] / G);
             const KeyT idle_inv = (KeyT)(a.idle_max - (G - C));
@@ -196,6 +211,7 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
         }
     }
     a.sortkey[(size_t)n * a.Hpad + h] = sk;
+    a.seq[(size_t)n * a.Hpad + h] = sq;
     a.feas[(size_t)n * a.Hpad + h] = f;
     PairT p;
     p.x = A;
@@ -296,6 +312,7 @@ Layout workspace_layout(int N, int Hpad)
     l.off_pk = o;      o = up(o + (size_t)N * Hpad * sizeof(uint4));
     l.off_tmp_feas = o; o = up(o + (size_t)N * Hpad * sizeof(int4));
     l.off_tmp_ab = o;  o = up(o + (size_t)N * Hpad * sizeof(ulonglong2));
+    l.off_tmp_seq = o; o = up(o + (size_t)N * Hpad * sizeof(int4));
     l.off_sortkey = o; o = up(o + (size_t)N * Hpad * sizeof(unsigned long long));
     l.off_perm = o;    o = up(o + (size_t)N * Hpad * sizeof(unsigned int));
     l.total = o;
@@ -441,7 +458,8 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     void *tmp_ab = ws + lay.off_tmp_ab;
     unsigned long long *sortkey = reinterpret_cast<unsigned long long *>(ws + lay.off_sortkey);
     unsigned int *perm = reinterpret_cast<unsigned int *>(ws + lay.off_perm);
-    EmitArgs ea{d_G, d_S, d_C, d_AV, d_AC, d_AM, d_limits, d_lambda, tmp_feas, tmp_ab, sortkey,
+    int4 *tmp_seq = reinterpret_cast<int4 *>(ws + lay.off_tmp_seq);
+    EmitArgs ea{d_G, d_S, d_C, d_AV, d_AC, d_AM, d_limits, d_lambda, tmp_feas, tmp_seq, tmp_ab, sortkey,
                 H, Hpad, s->R, s->flags, s->key_order, idle_max, k.bits_idle, k.bits_sr, k.bits_id};
     dim3 grid((Hpad + 255) / 256, N);
     if (k.key_bits == 32)
@@ -468,6 +486,9 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     s->d_feas = reinterpret_cast<const int4 *>(ws + lay.off_feas);
     s->d_ab = ws + lay.off_ab;
     s->d_pk = reinterpret_cast<const uint4 *>(ws + lay.off_pk);
+    s->d_host_feas = tmp_feas;
+    s->d_host_ab = tmp_ab;
+    s->d_host_seq = tmp_seq;
     return NBOS_OK;
 }
 

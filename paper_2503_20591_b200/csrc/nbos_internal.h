@@ -38,7 +38,7 @@ enum : unsigned int {
 
 struct Layout {
     size_t off_status, off_limits, off_sums, off_lambda, off_stats, off_feas, off_ab, off_pk;
-    size_t off_tmp_feas, off_tmp_ab, off_sortkey, off_perm, total;
+    size_t off_tmp_feas, off_tmp_ab, off_tmp_seq, off_sortkey, off_perm, total;
 };
 Layout workspace_layout(int n_snapshots, int hosts_padded);
 inline int pad_hosts(int h) { return (h + 31) & ~31; }
@@ -78,6 +78,10 @@ struct nbos_snapshot {
     const uint4 *d_pk;    // [N][Hpad] (word0, word1, A, B), only when pack.enabled
     nbos::PackLayout pack;
     int presorted;
+    // the same records in host-index order (what the derivation staged), for sequential placement
+    const int4 *d_host_feas;
+    const void *d_host_ab;
+    const int4 *d_host_seq;   // (min(G, idle GPUs), cap - S, S, 0)
     int device, sm_count;
     cudaStream_t owner_stream;  // stream the owned workspace was allocated on (create_host)
 };
@@ -104,6 +108,11 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
 int launch_place_static(const nbos_snapshot *s, const int32_t *d_requests, int64_t batch,
                         int32_t *d_out_hosts, int32_t *d_out_found, cudaStream_t stream,
                         int host_split);
+
+// Sequential placement with commits (nbos_sequential.cu).
+int launch_place_sequential(const nbos_snapshot *s, const int32_t *d_requests, int64_t batch,
+                            int32_t *d_out_hosts, int32_t *d_out_found, int32_t *d_out_subscribed,
+                            cudaStream_t stream);
 
 }  // namespace nbos
 #endif

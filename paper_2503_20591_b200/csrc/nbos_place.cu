@@ -46,7 +46,6 @@ enum : int {
 };
 __host__ __device__ constexpr bool mode_is_packed(int mode) { return mode >= MODE_PACKED; }
 __host__ __device__ constexpr bool mode_is_static(int mode) { return mode == MODE_PACKED_STATIC || mode == MODE_PACKED2_STATIC; }
-__host__ __device__ constexpr bool mode_two_masks(int mode) { return mode == MODE_PACKED2 || mode == MODE_PACKED2_STATIC; }
 __host__ __device__ constexpr int mode_record_bytes(int mode) { return mode == MODE_KEY64 ? 32 : mode == MODE_PLAIN ? 24 : 16; }
 __host__ __device__ constexpr int mode_max_q(int mode) { return mode == MODE_KEY64 ? 4 : 8; }
 constexpr int kStages = 3;

@@ -1,0 +1,233 @@
+// Sequential placement with commits (Sections 3.2.1, 3.4.1): requests of a snapshot are placed one
+// after the other, and a request that found three hosts adds its GPUs to their subscribed count
+// before the next request is looked at. The dependence is serial over requests, so the
+// parallelism is over hosts (all hosts of the snapshot are evaluated for one request at a time)
+// and over snapshots (one thread block each).
+//
+// One block of 1,024 threads owns a snapshot. Thread t owns hosts t, t + 1024, ...: the fields a
+// commit changes (room under the SR limit, key intercept A) live in registers, the static ones in
+// shared memory. Per request: every thread ranks its own hosts, each warp extracts its three
+// smallest keys with three warp-wide integer minimum reductions (keys are unique, the lane that
+// held the minimum pops it), warp 0 does the same over the 32 warps' triples, writes the result,
+// and the owners of the three winning hosts update them. Two block barriers per request.
+#include <limits.h>
+
+#include "nbos_internal.h"
+
+namespace nbos {
+namespace {
+
+constexpr int kSeqThreads = 1024;
+constexpr int kSeqWarps = kSeqThreads / 32;
+
+struct SeqParams {
+    const int4 *feas;   // [N][Hpad] host order: (gmax, vram, cpu, mem)
+    const void *ab;     // [N][Hpad] host order: (A, B)
+    const int4 *seq;    // [N][Hpad] host order: (min(G, idle), cap - S, S, 0)
+    const int4 *requests;
+    int32_t *out_hosts, *out_found, *out_subscribed;
+    long long B;
+    int H, Hpad;
+    unsigned int id_mask;
+};
+
+template <typename KeyT> struct SeqKey;
+template <> struct SeqKey<unsigned int> {
+    using Pair = uint2;
+    static constexpr unsigned int kInf = 0xFFFFFFFFu;
+    static __device__ __forceinline__ unsigned int warp_min(unsigned int k) { return __reduce_min_sync(0xFFFFFFFFu, k); }
+};
+template <> struct SeqKey<unsigned long long> {
+    using Pair = ulonglong2;
+    static constexpr unsigned long long kInf = 0xFFFFFFFFFFFFFFFFull;
+    static __device__ __forceinline__ unsigned long long warp_min(unsigned long long k)
+    {
+        const unsigned int hi = __reduce_min_sync(0xFFFFFFFFu, (unsigned int)(k >> 32));
+        const unsigned int lo = __reduce_min_sync(0xFFFFFFFFu, (unsigned int)(k >> 32) == hi ? (unsigned int)k : 0xFFFFFFFFu);
+        return ((unsigned long long)hi << 32) | lo;
+    }
+};
+
+template <typename KeyT>
+__device__ __forceinline__ void insert3(KeyT &t1, KeyT &t2, KeyT &t3, KeyT k)
+{
+    const KeyT hi1 = max(t1, k);
+    t1 = min(t1, k);
+    const KeyT hi2 = max(t2, hi1);
+    t2 = min(t2, hi1);
+    t3 = min(t3, hi2);
+}
+
+// The three smallest of the warp's keys (each lane brings a sorted triple); every lane returns them.
+template <typename KeyT>
+__device__ __forceinline__ void warp_best3(KeyT k1, KeyT k2, KeyT k3, KeyT &w1, KeyT &w2, KeyT &w3)
+{
+    constexpr KeyT kInf = SeqKey<KeyT>::kInf;
+    KeyT w[3];
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {
+        const KeyT m = SeqKey<KeyT>::warp_min(k1);
+        w[i] = m;
+        if (k1 == m && m != kInf) {  // unique keys: exactly one lane pops
+            k1 = k2;
+            k2 = k3;
+            k3 = kInf;
+        }
+    }
+    w1 = w[0]; w2 = w[1]; w3 = w[2];
+}
+
+// HPT = hosts per thread. Static per-host fields in shared memory: (vram, cpu, mem, g_cap) as int4
+// and B; dynamic in registers: room = cap - S, A, and the GPUs added so far.
+template <typename KeyT, int HPT>
+__global__ void __launch_bounds__(kSeqThreads, 1) place_sequential_kernel(const SeqParams p)
+{
+    using Pair = typename SeqKey<KeyT>::Pair;
+    constexpr KeyT kInf = SeqKey<KeyT>::kInf;
+    extern __shared__ __align__(16) unsigned char seq_smem[];
+    int4 *s_cap = reinterpret_cast<int4 *>(seq_smem);                                        // [HPT*1024]
+    KeyT *s_B = reinterpret_cast<KeyT *>(seq_smem + (size_t)HPT * kSeqThreads * sizeof(int4));  // [HPT*1024]
+    __shared__ KeyT s_warp[kSeqWarps][3];
+    __shared__ KeyT s_best[3];
+
+    const int n = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const size_t row = (size_t)n * p.Hpad;
+
+    int room[HPT], added[HPT];
+    KeyT A[HPT];
+#pragma unroll
+    for (int u = 0; u < HPT; ++u) {
+        const int h = tid + u * kSeqThreads;
+        int4 cap = make_int4(0, 0, 0, -1);
+        KeyT b = 0;
+        room[u] = -1;
+        added[u] = 0;
+        A[u] = kInf;
+        if (h < p.Hpad) {
+            const int4 f = p.feas[row + h];
+            const int4 sq = p.seq[row + h];
+            const Pair ab = reinterpret_cast<const Pair *>(p.ab)[row + h];
+            cap = make_int4(f.y, f.z, f.w, sq.x);
+            room[u] = sq.y;
+            // a host that takes nothing now has no key yet (A = h, B = 0): it can never take anything
+            // later either, because commits only shrink the room
+            A[u] = f.x >= 0 ? (KeyT)ab.x : kInf;
+            b = ab.y;
+            if (f.x < 0) room[u] = -1;
+        }
+        s_cap[h] = cap;
+        s_B[h] = b;
+    }
+    __syncthreads();
+
+    const int4 *req = p.requests + (size_t)n * p.B;
+    int4 next = p.B > 0 ? __ldg(req) : make_int4(-1, 0, 0, 0);
+    for (long long r = 0; r < p.B; ++r) {
+        const int4 q = next;
+        if (r + 1 < p.B) next = __ldg(req + r + 1);
+        const bool sane = (q.x | q.y | q.z | q.w) >= 0;
+        KeyT k1 = kInf, k2 = kInf, k3 = kInf;
+        if (sane) {
+#pragma unroll
+            for (int u = 0; u < HPT; ++u) {
+                const int h = tid + u * kSeqThreads;
+                const int4 cap = s_cap[h];
+                const bool ok = q.x <= min(cap.w, room[u]) && q.y <= cap.x && q.z <= cap.y && q.w <= cap.z;
+                const KeyT key = ok ? (KeyT)(A[u] + (KeyT)(unsigned int)q.x * s_B[h]) : kInf;
+                insert3(k1, k2, k3, key);
+            }
+        }
+        KeyT w1, w2, w3;
+        warp_best3(k1, k2, k3, w1, w2, w3);
+        if (lane == 0) {
+            s_warp[warp][0] = w1;
+            s_warp[warp][1] = w2;
+            s_warp[warp][2] = w3;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            KeyT b1, b2, b3;
+            warp_best3(s_warp[lane][0], s_warp[lane][1], s_warp[lane][2], b1, b2, b3);
+            if (lane == 0) {
+                s_best[0] = b1;
+                s_best[1] = b2;
+                s_best[2] = b3;
+                const long long o = (long long)n * p.B + r;
+                p.out_hosts[o * 3 + 0] = b1 == kInf ? -1 : (int)((unsigned int)b1 & p.id_mask);
+                p.out_hosts[o * 3 + 1] = b2 == kInf ? -1 : (int)((unsigned int)b2 & p.id_mask);
+                p.out_hosts[o * 3 + 2] = b3 == kInf ? -1 : (int)((unsigned int)b3 & p.id_mask);
+                if (p.out_found) p.out_found[o] = (b1 != kInf) + (b2 != kInf) + (b3 != kInf);
+            }
+        }
+        __syncthreads();
+        // commit: only a kernel that got all three replicas is created
+        if (s_best[2] != kInf && q.x > 0) {
+#pragma unroll
+            for (int i = 0; i < 3; ++i) {
+                const int h = (int)((unsigned int)s_best[i] & p.id_mask);
+                if ((h & (kSeqThreads - 1)) == tid) {
+                    const int u0 = h / kSeqThreads;
+#pragma unroll
+                    for (int u = 0; u < HPT; ++u)
+                        if (u == u0) {
+                            room[u] -= q.x;
+                            added[u] += q.x;
+                            A[u] += (KeyT)(unsigned int)q.x * s_B[h];
+                        }
+                }
+            }
+        }
+        // s_best is rewritten only after the next request's first barrier, which every thread
+        // reaches after having read it here
+    }
+    if (p.out_subscribed) {
+#pragma unroll
+        for (int u = 0; u < HPT; ++u) {
+            const int h = tid + u * kSeqThreads;
+            if (h < p.H) p.out_subscribed[(size_t)n * p.H + h] = p.seq[row + h].z + added[u];
+        }
+    }
+}
+
+template <typename KeyT>
+int launch_seq(const SeqParams &p, int N, int hpt, cudaStream_t stream)
+{
+    const size_t smem = (size_t)hpt * kSeqThreads * (sizeof(int4) + sizeof(KeyT));
+    void (*fn)(const SeqParams) = hpt == 1 ? place_sequential_kernel<KeyT, 1>
+                                  : hpt == 2 ? place_sequential_kernel<KeyT, 2>
+                                  : hpt == 4 ? place_sequential_kernel<KeyT, 4>
+                                             : place_sequential_kernel<KeyT, 8>;
+    NBOS_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    fn<<<N, kSeqThreads, smem, stream>>>(p);
+    NBOS_CUDA_TRY(cudaGetLastError());
+    return NBOS_OK;
+}
+
+}  // namespace
+
+int launch_place_sequential(const nbos_snapshot *s, const int32_t *d_requests, int64_t batch,
+                            int32_t *d_out_hosts, int32_t *d_out_found, int32_t *d_out_subscribed,
+                            cudaStream_t stream)
+{
+    SeqParams p;
+    p.feas = s->d_host_feas;
+    p.ab = s->d_host_ab;
+    p.seq = s->d_host_seq;
+    p.requests = reinterpret_cast<const int4 *>(d_requests);
+    p.out_hosts = d_out_hosts;
+    p.out_found = d_out_found;
+    p.out_subscribed = d_out_subscribed;
+    p.B = batch;
+    p.H = s->H;
+    p.Hpad = s->Hpad;
+    p.id_mask = (1u << s->key.bits_id) - 1u;
+    if (batch == 0 && !d_out_subscribed) return NBOS_OK;
+    int hpt = 1;
+    while (hpt * kSeqThreads < s->Hpad) hpt <<= 1;
+    if (hpt > 8) return fail(NBOS_ERR_RANGE, "sequential placement supports at most %d hosts", NBOS_SEQUENTIAL_MAX_HOSTS);
+    return s->key.key_bits == 64 ? launch_seq<unsigned long long>(p, s->N, hpt, stream)
+                                 : launch_seq<unsigned int>(p, s->N, hpt, stream);
+}
+
+}  // namespace nbos
