@@ -434,6 +434,28 @@ def run_ours(args):
             "designated": int((ex >= 0).sum().item()), "all_yield": int((ex < 0).sum().item()),
             "note": "inputs + outputs 576 MiB, larger than L2"}
 
+        # sequential placement with commits: serial over requests, parallel over hosts / snapshots
+        for label, ww in (("sequential_cfg4_shape", W.make_config(4)),
+                          ("sequential_one_snapshot_4096_hosts", W.make_config(3, batch=65_536))):
+            sn = nb.snapshot_from_workload(ww, device=dev, flags=nb.NBOS_ROOM_FOR_COMMITS)
+            rq = torch.from_numpy(ww.requests).to(dev)
+            oh = torch.empty((ww.n_snapshots, ww.batch, 3), dtype=torch.int32, device=dev)
+            of = torch.empty((ww.n_snapshots, ww.batch), dtype=torch.int32, device=dev)
+            nb.nbos_place_batch_sequential(sn, rq, oh, of, stream=stream)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(3):
+                nb.nbos_place_batch_sequential(sn, rq, oh, of, stream=stream)
+            b.record(stream)
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / 3
+            others[label] = {"n_snapshots": ww.n_snapshots, "n_hosts": ww.n_hosts, "batch": ww.batch,
+                             "kernel_ms": ms, "decisions_per_s": ww.decisions / ms * 1e3,
+                             "us_per_request_per_snapshot": ms * 1e3 / ww.batch,
+                             "kernels_created": int((of == 3).sum().item())}
+            nb.nbos_snapshot_destroy(sn)
+
     rot_mib = n_rot * per_batch_bytes / 2**20
     launches_per_step = 5  # scan, emit, rank, finalize (derivation) + placement kernel
     line = {
