@@ -174,9 +174,10 @@ int nbos_snapshot_create(const nbos_snapshot_desc *desc, void *workspace, size_t
                          void *cuda_stream, nbos_snapshot **out);
 
 /* Same operation from HOST arrays (any alignment). The library takes the workspace and a staging
- * buffer from the device's stream-ordered memory pool (cudaMallocAsync on `cuda_stream`) and
- * returns them in nbos_snapshot_destroy / when the derivation has run. The host arrays have been
- * read when the call returns. */
+ * buffer from a stream-ordered memory pool of its own (one per device, kept for the life of the
+ * process so that repeated calls reuse the same memory) and gives them back to that pool in
+ * nbos_snapshot_destroy / when the derivation has run. The host arrays have been read when the
+ * call returns. */
 int nbos_snapshot_create_host(const nbos_snapshot_desc *desc, void *cuda_stream,
                               nbos_snapshot **out);
 
@@ -210,7 +211,7 @@ int nbos_place_batch_ex(const nbos_snapshot *snap, const int32_t *requests,
  * Same operation with HOST buffers (pinned memory makes the copies asynchronous and faster, but
  * any host memory works). The batch is cut into up to 16 chunks whose host-to-device copy, kernel
  * and device-to-host copy overlap on three internal streams (created once per device; calls on
- * the same device take turns). Device staging comes from the stream-ordered memory pool. Returns
+ * the same device take turns). Device staging comes from the library's own memory pool. Returns
  * after the results are in the host buffers.
  */
 int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_host,

@@ -87,6 +87,10 @@ struct HostPipe {
     bool ready = false;
     cudaStream_t streams[kStreams] = {};
     cudaEvent_t start = nullptr, done[kStreams] = {};
+    // The library's own stream-ordered pool for staging buffers. Its release threshold is
+    // unlimited, so the buffers of one call are reused by the next instead of going back to the
+    // driver at every synchronisation (which costs more than the placement itself).
+    cudaMemPool_t pool = nullptr;
 };
 HostPipe g_pipes[64];
 std::mutex g_pipes_mutex;
@@ -102,6 +106,14 @@ int host_pipe(int device, HostPipe **out)
             NBOS_CUDA_TRY(cudaEventCreateWithFlags(&p.done[j], cudaEventDisableTiming));
         }
         NBOS_CUDA_TRY(cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming));
+        cudaMemPoolProps props = {};
+        props.allocType = cudaMemAllocationTypePinned;
+        props.handleTypes = cudaMemHandleTypeNone;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = device;
+        NBOS_CUDA_TRY(cudaMemPoolCreate(&p.pool, &props));
+        unsigned long long keep = ~0ull;
+        NBOS_CUDA_TRY(cudaMemPoolSetAttribute(p.pool, cudaMemPoolAttrReleaseThreshold, &keep));
         p.ready = true;
     }
     *out = &p;
@@ -187,9 +199,12 @@ int nbos_snapshot_create_host(const nbos_snapshot_desc *desc, void *cuda_stream,
     const size_t cells = (size_t)desc->n_snapshots * desc->n_hosts;
     const size_t arr_bytes = (cells * sizeof(int32_t) + 255) & ~(size_t)255;
     const size_t need = workspace_layout(desc->n_snapshots, pad_hosts(desc->n_hosts)).total;
+    HostPipe *pipe = nullptr;
+    rc = host_pipe(device, &pipe);
+    if (rc) return rc;
     void *ws = nullptr, *staging = nullptr;
-    cudaError_t e = cudaMallocAsync(&ws, need, stream);
-    if (e == cudaSuccess) e = cudaMallocAsync(&staging, 6 * arr_bytes, stream);
+    cudaError_t e = cudaMallocFromPoolAsync(&ws, need, pipe->pool, stream);
+    if (e == cudaSuccess) e = cudaMallocFromPoolAsync(&staging, 6 * arr_bytes, pipe->pool, stream);
     if (e != cudaSuccess) {
         if (ws) cudaFreeAsync(ws, stream);
         cudaGetLastError();
@@ -304,7 +319,7 @@ int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_hos
     std::lock_guard<std::mutex> lock(pipe->mutex);
 
     char *buf = nullptr;
-    cudaError_t e = cudaMallocAsync(reinterpret_cast<void **>(&buf), up(req_bytes) + up(out_bytes) + up(found_bytes), stream);
+    cudaError_t e = cudaMallocFromPoolAsync(reinterpret_cast<void **>(&buf), up(req_bytes) + up(out_bytes) + up(found_bytes), pipe->pool, stream);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return fail(NBOS_ERR_NO_MEMORY, "device staging allocation failed: %s", cudaGetErrorString(e));
@@ -315,10 +330,20 @@ int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_hos
 
     // chunks of the flattened request list: copy in, place, copy out, round-robin over the side
     // streams so that the copies of one chunk overlap the kernel of another
-    long long n_chunks = total / (128 * 1024);
-    if (n_chunks < 1) n_chunks = 1;
-    if (n_chunks > 16) n_chunks = 16;
-    const long long chunk = ((total + n_chunks - 1) / n_chunks + 31) & ~31ll;
+    // chunk = a whole number of full passes of all resident blocks (so that the lanes of every chunk
+    // launch are as busy as in a single launch), about six chunks
+    int lanes = 0;
+    long long unit = 0;
+    rc = place_chunk_unit(snap, total, &lanes, &unit);
+    if (rc) {
+        cudaFreeAsync(buf, stream);
+        return rc;
+    }
+    long long passes = total / unit;            // full passes in the batch
+    long long per_chunk = passes >= 12 ? passes / 6 : passes >= 4 ? 1 : 0;
+    const long long chunk = per_chunk ? per_chunk * unit : ((total + 31) & ~31ll);
+    nbos_launch_config chunk_cfg = {};
+    chunk_cfg.lanes_per_request = lanes;
     e = cudaEventRecord(pipe->start, stream);
     for (int j = 0; j < HostPipe::kStreams && e == cudaSuccess; ++j) e = cudaStreamWaitEvent(pipe->streams[j], pipe->start, 0);
     int used = 0;
@@ -328,7 +353,7 @@ int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_hos
         if (i < HostPipe::kStreams) used = (int)i + 1;
         e = cudaMemcpyAsync(d_req + lo * 4, requests_host + lo * 4, (size_t)n * 16, cudaMemcpyHostToDevice, st);
         if (e != cudaSuccess) break;
-        rc = launch_place(snap, d_req, batch_per_snapshot, d_out, d_found, st, nullptr, lo, n);
+        rc = launch_place(snap, d_req, batch_per_snapshot, d_out, d_found, st, &chunk_cfg, lo, n);
         if (rc) break;
         e = cudaMemcpyAsync(out_hosts_host + lo * 3, d_out + lo * 3, (size_t)n * 12, cudaMemcpyDeviceToHost, st);
         if (e == cudaSuccess && d_found)

@@ -744,7 +744,83 @@ void fill_params(PlaceParams &p, const nbos_snapshot *s, const int32_t *d_reques
 
 bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
 
+
+// What launch_place decides before it looks at the host split: evaluation mode, tile size,
+// shared memory, resident blocks per SM and lanes per request.
+struct LaunchPlan {
+    int mode, T, tiles_total, per_sm, L;
+    size_t smem;
+};
+
+int make_plan(const nbos_snapshot *s, long long total, const nbos_launch_config &c, LaunchPlan &plan)
+{
+    const int mode = snapshot_mode(s, c.pair_mode);
+    const int record = mode_record_bytes(mode);
+    const int max_q_kernel = mode_max_q(mode);
+
+    // tile: as many hosts as fit the stage budget, at most the whole (padded) table
+    int T = c.tile_hosts ? c.tile_hosts : 1024;
+    if (T > s->Hpad) T = s->Hpad;
+    const int max_tile = (64 * 1024) / record / 32 * 32;  // <= 64 KB per stage
+    if (T > max_tile) T = max_tile;
+    const int tiles_total = (s->Hpad + T - 1) / T;
+
+    KernelFn fn1 = pick_kernel(mode, 1);
+    const size_t smem = (size_t)kStages * T * record + 2 * kStages * 8 + 16;
+    NBOS_CUDA_TRY(cudaFuncSetAttribute(fn1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    int per_sm = 0;
+    NBOS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn1, kThreads, smem));
+    if (per_sm < 1) return fail(NBOS_ERR_CUDA, "placement kernel does not fit on an SM (%zu bytes of shared memory)", smem);
+
+    // Lanes per request: estimate, for each L, the pair steps one lane of the busiest block has to
+    // make (passes in units of requests per lane, weighted by how well a pass of that size
+    // amortises the per-host overhead, times hosts per lane) plus the shuffle merges, and take
+    // the cheapest. Large batches end up with few lanes, small ones with a whole warp.
+    int L = c.lanes_per_request;
+    if (!L) {
+        const long long slots = (long long)s->sm_count * per_sm;
+        double best = 0.0;
+        for (int cand = 1, lg = 0; cand <= 32; cand <<= 1, ++lg) {
+            const long long groups = kComputeThreads / cand;
+            long long ctas = (total + groups - 1) / groups;
+            if (ctas > slots) ctas = slots;
+            const long long n_req = (total + ctas - 1) / ctas;
+            const long long full = n_req / (groups * max_q_kernel), rem = n_req % (groups * max_q_kernel);
+            int q = max_q_kernel;
+            while (q > 2 && (long long)(q >> 1) * groups >= rem) q >>= 1;
+            const double weight = q >= 8 ? 1.0 : q == 4 ? 1.12 : 1.4;
+            const double units = (double)full * max_q_kernel + (rem ? q * weight : 0.0);
+            const double cost = units * ((double)s->Hpad / cand) + (double)(full + (rem ? 1 : 0)) * lg * max_q_kernel * 4.0;
+            if (cand == 1 || cost < best * 0.98) {
+                best = cost;
+                L = cand;
+            }
+        }
+    }
+    plan.mode = mode;
+    plan.T = T;
+    plan.tiles_total = tiles_total;
+    plan.per_sm = per_sm;
+    plan.L = L;
+    plan.smem = smem;
+    return NBOS_OK;
+}
+
 }  // namespace
+
+// For callers that cut a batch into several launches (the host-buffer pipeline): the lanes per
+// request the whole batch would get, and the number of requests that gives every resident block
+// exactly one full pass -- chunks that are multiples of it keep every lane busy.
+int place_chunk_unit(const nbos_snapshot *s, long long total, int *lanes, long long *unit)
+{
+    nbos_launch_config c = {};
+    LaunchPlan plan;
+    int rc = make_plan(s, total, c, plan);
+    if (rc) return rc;
+    *lanes = plan.L;
+    *unit = (long long)s->sm_count * plan.per_sm * (kComputeThreads / plan.L) * mode_max_q(plan.mode);
+    return NBOS_OK;
+}
 
 int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batch,
                  int32_t *d_out_hosts, int32_t *d_out_found, cudaStream_t stream,
@@ -789,51 +865,15 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
         return NBOS_OK;
     }
 
-    const int mode = snapshot_mode(s, c.pair_mode);
-    const bool k64 = mode == MODE_KEY64;
-    const int record = mode_record_bytes(mode);
+    LaunchPlan plan;
+    int rc = make_plan(s, total, c, plan);
+    if (rc) return rc;
+    const int mode = plan.mode, T = plan.T, tiles_total = plan.tiles_total, L = plan.L;
     const int max_q_kernel = mode_max_q(mode);
-
-    // tile: as many hosts as fit the stage budget, at most the whole (padded) table
-    int T = c.tile_hosts ? c.tile_hosts : 1024;
-    if (T > s->Hpad) T = s->Hpad;
-    const int max_tile = (64 * 1024) / record / 32 * 32;  // <= 64 KB per stage
-    if (T > max_tile) T = max_tile;
-    const int tiles_total = (s->Hpad + T - 1) / T;
-
-    KernelFn fn1 = pick_kernel(mode, 1);
-    const size_t smem = (size_t)kStages * T * record + 2 * kStages * 8 + 16;
-    NBOS_CUDA_TRY(cudaFuncSetAttribute(fn1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    int per_sm = 0;
-    NBOS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn1, kThreads, smem));
-    if (per_sm < 1) return fail(NBOS_ERR_CUDA, "placement kernel does not fit on an SM (%zu bytes of shared memory)", smem);
-
-    // Lanes per request: estimate, for each L, the pair steps one lane of the busiest block has to
-    // make (passes in units of requests per lane, weighted by how well a pass of that size
-    // amortises the per-host overhead, times hosts per lane) plus the shuffle merges, and take
-    // the cheapest. Large batches end up with few lanes, small ones with a whole warp.
+    const bool k64 = mode == MODE_KEY64;
+    const size_t smem = plan.smem;
+    int per_sm = plan.per_sm;
     const long long want_threads = (long long)s->sm_count * per_sm * kComputeThreads;
-    int L = c.lanes_per_request;
-    if (!L) {
-        const long long slots = (long long)s->sm_count * per_sm;
-        double best = 0.0;
-        for (int cand = 1, lg = 0; cand <= 32; cand <<= 1, ++lg) {
-            const long long groups = kComputeThreads / cand;
-            long long ctas = (total + groups - 1) / groups;
-            if (ctas > slots) ctas = slots;
-            const long long n_req = (total + ctas - 1) / ctas;
-            const long long full = n_req / (groups * max_q_kernel), rem = n_req % (groups * max_q_kernel);
-            int q = max_q_kernel;
-            while (q > 2 && (long long)(q >> 1) * groups >= rem) q >>= 1;
-            const double weight = q >= 8 ? 1.0 : q == 4 ? 1.12 : 1.4;
-            const double units = (double)full * max_q_kernel + (rem ? q * weight : 0.0);
-            const double cost = units * ((double)s->Hpad / cand) + (double)(full + (rem ? 1 : 0)) * lg * max_q_kernel * 4.0;
-            if (cand == 1 || cost < best * 0.98) {
-                best = cost;
-                L = cand;
-            }
-        }
-    }
     int K = c.host_split;
     if (!K) {
         K = 1;
