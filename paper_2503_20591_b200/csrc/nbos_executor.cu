@@ -52,15 +52,28 @@ __global__ void __launch_bounds__(512) select_executors_kernel(const ExecArgs a)
         fit = s_fit;
         rank = s_rank;
     }
-    for (long long k = (long long)blockIdx.x * blockDim.x + threadIdx.x; k < a.n_kernels;
-         k += (long long)gridDim.x * blockDim.x) {
-        const int4 r = __ldg(a.requests + k);
+    // the streams of the next iteration are requested before this iteration's records are
+    // gathered, so that every thread always has a request and three host ids in flight
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    long long k = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    int4 r_next = make_int4(-1, 0, 0, 0);
+    int h_next[3] = {-1, -1, -1};
+    if (k < a.n_kernels) {
+        r_next = __ldg(a.requests + k);
+#pragma unroll
+        for (int slot = 0; slot < 3; ++slot) h_next[slot] = __ldg(a.replica_hosts + 3 * k + slot);
+    }
+    for (; k < a.n_kernels; k += stride) {
+        const int4 r = r_next;
+        int h[3] = {h_next[0], h_next[1], h_next[2]};
+        if (k + stride < a.n_kernels) {
+            r_next = __ldg(a.requests + k + stride);
+#pragma unroll
+            for (int slot = 0; slot < 3; ++slot) h_next[slot] = __ldg(a.replica_hosts + 3 * (k + stride) + slot);
+        }
         const bool sane = (r.x | r.y | r.z | r.w) >= 0;
-        int h[3];
         int4 f[3];
         bool ok[3];
-#pragma unroll
-        for (int slot = 0; slot < 3; ++slot) h[slot] = __ldg(a.replica_hosts + 3 * k + slot);
 #pragma unroll
         for (int slot = 0; slot < 3; ++slot) {
             const bool valid = sane && h[slot] >= 0 && h[slot] < a.H;
@@ -72,29 +85,32 @@ __global__ void __launch_bounds__(512) select_executors_kernel(const ExecArgs a)
         if (mask != 0 && (mask & (mask - 1)) == 0) {
             best = ok[0] ? h[0] : ok[1] ? h[1] : h[2];  // a single runnable replica: no ranking needed
         } else if (mask != 0) {
-            long long best_idle = 0, best_S = 0, best_G = 1;
+            int best_idle = 0, best_slot = 0;
+            int2 best_gs = make_int2(1, 0);
+            bool have_gs = false;  // (G, S) of the current best is fetched only when idle GPUs tie
 #pragma unroll
             for (int slot = 0; slot < 3; ++slot) {
                 if (!ok[slot]) continue;
-                const int2 gs = rank[h[slot]];
-                const long long idle = f[slot].x, G = gs.x, S = gs.y;
-                bool before = best < 0;
-                if (!before) {
-                    if (idle != best_idle) {
-                        before = idle > best_idle;
-                    } else {
-                        // S / (G R) against best_S / (best_G R): R cancels, cross-multiply exactly
-                        const long long lhs = S * best_G, rhs = best_S * G;
-                        before = lhs != rhs ? lhs < rhs : h[slot] < best;
-                    }
+                const int idle = f[slot].x;
+                bool before = best < 0 || idle > best_idle;
+                if (best >= 0 && idle == best_idle) {
+                    if (!have_gs) best_gs = rank[best];
+                    const int2 gs = rank[h[slot]];
+                    // S / (G R) against best_S / (best_G R): R cancels, cross-multiply exactly
+                    const long long lhs = (long long)gs.y * best_gs.x, rhs = (long long)best_gs.y * gs.x;
+                    before = lhs != rhs ? lhs < rhs : h[slot] < best;
+                    if (before) best_gs = gs;
+                    have_gs = true;
+                } else if (before) {
+                    have_gs = false;
                 }
                 if (before) {
                     best = h[slot];
                     best_idle = idle;
-                    best_S = S;
-                    best_G = G;
+                    best_slot = slot;
                 }
             }
+            (void)best_slot;
         }
         a.out_executor[k] = best;
         a.out_can_run[k] = mask;
