@@ -35,7 +35,7 @@ ALGORITHMIC_OPS_PER_PAIR = 6      # 4 capacity compares + 1 multiply-add (key) +
 L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (read + write) of one placement-kernel launch on the default workload, from the ncu
 # capture summarised under profiles/. None while no capture matches the current kernel.
-PLACE_KERNEL_DRAM_BYTES_PER_LAUNCH = 16_914_176  # profiles/place_kernel_cfg3_launch_list.md
+PLACE_KERNEL_DRAM_BYTES_PER_LAUNCH = 16_914_176
 
 
 def parse_args():

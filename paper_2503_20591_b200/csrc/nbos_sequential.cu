@@ -8,8 +8,10 @@
 // commit changes (room under the SR limit, key intercept A) live in registers, the static ones in
 // shared memory. Per request: every thread ranks its own hosts, each warp extracts its three
 // smallest keys with three warp-wide integer minimum reductions (keys are unique, the lane that
-// held the minimum pops it), warp 0 does the same over the 32 warps' triples, writes the result,
+// held the minimum pops it), warp 0 does the same over the warps' triples, writes the result,
 // and the owners of the three winning hosts update them. Two block barriers per request.
+// (512 threads with twice the hosts each were measured slower: the per-thread chain of
+// best-three insertions is the critical path, not the per-warp reduction cost.)
 #include <limits.h>
 
 #include "nbos_internal.h"
@@ -77,7 +79,7 @@ __device__ __forceinline__ void warp_best3(KeyT k1, KeyT k2, KeyT k3, KeyT &w1, 
     w1 = w[0]; w2 = w[1]; w3 = w[2];
 }
 
-// HPT = hosts per thread. Static per-host fields in shared memory: (vram, cpu, mem, g_cap) as int4
+// HPT = hosts per thread (1..8). Static per-host fields in shared memory: (vram, cpu, mem, g_cap) as int4
 // and B; dynamic in registers: room = cap - S, A, and the GPUs added so far.
 template <typename KeyT, int HPT>
 __global__ void __launch_bounds__(kSeqThreads, 1) place_sequential_kernel(const SeqParams p)
@@ -94,7 +96,7 @@ __global__ void __launch_bounds__(kSeqThreads, 1) place_sequential_kernel(const 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const size_t row = (size_t)n * p.Hpad;
 
-    int room[HPT], added[HPT];
+    int gmax_now[HPT], room[HPT], added[HPT];  // gmax_now = min(g_cap, room): largest ask that fits now
     KeyT A[HPT];
 #pragma unroll
     for (int u = 0; u < HPT; ++u) {
@@ -116,6 +118,7 @@ __global__ void __launch_bounds__(kSeqThreads, 1) place_sequential_kernel(const 
             b = ab.y;
             if (f.x < 0) room[u] = -1;
         }
+        gmax_now[u] = min(cap.w, room[u]);
         s_cap[h] = cap;
         s_B[h] = b;
     }
@@ -133,7 +136,7 @@ __global__ void __launch_bounds__(kSeqThreads, 1) place_sequential_kernel(const 
             for (int u = 0; u < HPT; ++u) {
                 const int h = tid + u * kSeqThreads;
                 const int4 cap = s_cap[h];
-                const bool ok = q.x <= min(cap.w, room[u]) && q.y <= cap.x && q.z <= cap.y && q.w <= cap.z;
+                const bool ok = q.x <= gmax_now[u] && q.y <= cap.x && q.z <= cap.y && q.w <= cap.z;
                 const KeyT key = ok ? (KeyT)(A[u] + (KeyT)(unsigned int)q.x * s_B[h]) : kInf;
                 insert3(k1, k2, k3, key);
             }
@@ -148,7 +151,8 @@ __global__ void __launch_bounds__(kSeqThreads, 1) place_sequential_kernel(const 
         __syncthreads();
         if (warp == 0) {
             KeyT b1, b2, b3;
-            warp_best3(s_warp[lane][0], s_warp[lane][1], s_warp[lane][2], b1, b2, b3);
+            const bool has = lane < kSeqWarps;
+            warp_best3(has ? s_warp[lane][0] : kInf, has ? s_warp[lane][1] : kInf, has ? s_warp[lane][2] : kInf, b1, b2, b3);
             if (lane == 0) {
                 s_best[0] = b1;
                 s_best[1] = b2;
@@ -172,6 +176,7 @@ __global__ void __launch_bounds__(kSeqThreads, 1) place_sequential_kernel(const 
                     for (int u = 0; u < HPT; ++u)
                         if (u == u0) {
                             room[u] -= q.x;
+                            gmax_now[u] = min(s_cap[h].w, room[u]);
                             added[u] += q.x;
                             A[u] += (KeyT)(unsigned int)q.x * s_B[h];
                         }
