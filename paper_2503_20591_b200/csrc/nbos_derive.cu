@@ -18,6 +18,7 @@ namespace {
 struct ScanArgs {
     const int32_t *G, *S, *C, *AV, *AC, *AM;
     const longlong2 *limits;  // per snapshot (num * R, den): cap = floor(limits.x * G / limits.y)
+    longlong2 limit0;         // used instead of limits[0] when `limits` is null (single snapshot)
     SnapStats *stats;
     int H, R, flags;
 };
@@ -103,7 +104,7 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
         s_sub_max = 0ull;
     }
     __syncthreads();
-    const longlong2 lim = a.limits[n];
+    const longlong2 lim = a.limits ? a.limits[n] : a.limit0;
     unsigned int err = 0u;
     int idle_max = 0, g_min_inv = 0;  // INT_MAX - smallest G seen, 0 = none
     unsigned long long sub_max = 0ull;
@@ -159,7 +160,9 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
 struct EmitArgs {
     const int32_t *G, *S, *C, *AV, *AC, *AM;
     const longlong2 *limits;
-    const long long *lambda;  // per snapshot
+    longlong2 limit0;         // used when `limits` is null (single snapshot)
+    const long long *lambda;  // per snapshot; null = every host has w = 1 (one GPU count per snapshot)
+    unsigned int *rank;       // [N][Hpad], cleared here for rank_kernel (null = no visiting order)
     int4 *feas;                 // records in host-index order (staging)
     int4 *seq;                  // (min(G, idle), cap - S, S, 0) per host, for sequential placement
     void *ab;
@@ -186,7 +189,7 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
     if (h < a.H) {
         const size_t i = (size_t)n * a.H + h;
         const int G = a.G[i], S = a.S[i], C = a.C[i];
-        const longlong2 lim = a.limits[n];
+        const longlong2 lim = a.limits ? a.limits[n] : a.limit0;
         const int gm = derive_gmax(G, S, C, lim.x, lim.y, a.flags);
         f = make_int4(gm, a.AV[i], a.AC[i], a.AM[i]);
         sq.z = S;
@@ -197,7 +200,7 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
             sq = make_int4(g_cap, (int)room, S, 0);
         }
         if (gm >= 0) {
-            const KeyT w = (KeyT)(a.lambda[n] / G);
+            const KeyT w = a.lambda ? (KeyT)(a.lambda[n] / G) : (KeyT)1;
             const KeyT idle_inv = (KeyT)(a.idle_max - (G - C));
             const KeyT sr0 = (KeyT)S * w;
             if (a.key_order == NBOS_KEY_SR_FIRST) {
@@ -212,6 +215,7 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
     }
     a.sortkey[(size_t)n * a.Hpad + h] = sk;
     a.seq[(size_t)n * a.Hpad + h] = sq;
+    if (a.rank) a.rank[(size_t)n * a.Hpad + h] = 0u;
     a.feas[(size_t)n * a.Hpad + h] = f;
     PairT p;
     p.x = A;
@@ -365,12 +369,15 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
         sums_kernel<<<dim3(bx, N), 256, 0, stream>>>(d_G, d_S, d_C, H, d_sums);
         limits_from_sums_kernel<<<(N + 255) / 256, 256, 0, stream>>>(d_sums, d_limits, N);
         NBOS_CUDA_TRY(cudaGetLastError());
-    } else {
+    } else if (N > 1) {
         NBOS_CUDA_TRY(cudaMemcpyAsync(d_limits, h_limits, sizeof(longlong2) * (size_t)N,
                                       cudaMemcpyHostToDevice, stream));
     }
+    // a single snapshot's fixed limit travels in the kernel arguments instead of a copy
+    const longlong2 *limits_arg = (N == 1 && !dynamic_limit) ? nullptr : d_limits;
+    const longlong2 limit0 = (N == 1 && !dynamic_limit) ? h_limits[0] : make_longlong2(0, 1);
 
-    ScanArgs sa{d_G, d_S, d_C, d_AV, d_AC, d_AM, d_limits, d_stats, H, s->R, s->flags};
+    ScanArgs sa{d_G, d_S, d_C, d_AV, d_AC, d_AM, limits_arg, limit0, d_stats, H, s->R, s->flags};
     scan_kernel<<<dim3(bx, N), 256, 0, stream>>>(sa);
     NBOS_CUDA_TRY(cudaGetLastError());
     NBOS_CUDA_TRY(cudaMemcpyAsync(h_stats, d_stats, sizeof(SnapStats) * (size_t)N,
@@ -452,14 +459,17 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     }
     s->pack = pk;
 
-    NBOS_CUDA_TRY(cudaMemcpyAsync(d_lambda, h_lambda, sizeof(long long) * (size_t)N,
-                                  cudaMemcpyHostToDevice, stream));
+    if (!k.static_key)
+        NBOS_CUDA_TRY(cudaMemcpyAsync(d_lambda, h_lambda, sizeof(long long) * (size_t)N,
+                                      cudaMemcpyHostToDevice, stream));
+    s->presorted = Hpad <= kSortMaxHosts;
     int4 *tmp_feas = reinterpret_cast<int4 *>(ws + lay.off_tmp_feas);
     void *tmp_ab = ws + lay.off_tmp_ab;
     unsigned long long *sortkey = reinterpret_cast<unsigned long long *>(ws + lay.off_sortkey);
     unsigned int *perm = reinterpret_cast<unsigned int *>(ws + lay.off_perm);
     int4 *tmp_seq = reinterpret_cast<int4 *>(ws + lay.off_tmp_seq);
-    EmitArgs ea{d_G, d_S, d_C, d_AV, d_AC, d_AM, d_limits, d_lambda, tmp_feas, tmp_seq, tmp_ab, sortkey,
+    EmitArgs ea{d_G, d_S, d_C, d_AV, d_AC, d_AM, limits_arg, limit0, k.static_key ? nullptr : d_lambda,
+                s->presorted ? perm : nullptr, tmp_feas, tmp_seq, tmp_ab, sortkey,
                 H, Hpad, s->R, s->flags, s->key_order, idle_max, k.bits_idle, k.bits_sr, k.bits_id};
     dim3 grid((Hpad + 255) / 256, N);
     if (k.key_bits == 32)
@@ -469,9 +479,7 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     NBOS_CUDA_TRY(cudaGetLastError());
 
     // visiting order
-    s->presorted = Hpad <= kSortMaxHosts;
     if (s->presorted) {
-        NBOS_CUDA_TRY(cudaMemsetAsync(perm, 0, sizeof(unsigned int) * (size_t)N * Hpad, stream));
         rank_kernel<<<dim3((Hpad + 255) / 256, (Hpad + kRankChunk - 1) / kRankChunk, N), 256, 0, stream>>>(sortkey, perm, Hpad);
         NBOS_CUDA_TRY(cudaGetLastError());
     }
