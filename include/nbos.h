@@ -57,6 +57,8 @@ extern "C" {
 #define NBOS_ERR_UNSUPPORTED_DEVICE (-4) /* current device is not compute capability 10.x       */
 #define NBOS_ERR_DEVICE_TIMEOUT (-5)     /* a bounded wait inside a kernel ran out              */
 #define NBOS_ERR_NO_MEMORY (-6)          /* host or device allocation failed / workspace small  */
+#define NBOS_ERR_STALE_LAYOUT (-7)       /* nbos_snapshot_update: new state does not fit the key /
+                                          * packing layout chosen at creation; create a new one  */
 
 /* key_order */
 #define NBOS_KEY_IDLE_FIRST 0 /* Section 3.4.1: idle GPUs, then SR, then host id (default) */
@@ -180,6 +182,28 @@ int nbos_snapshot_create(const nbos_snapshot_desc *desc, void *workspace, size_t
  * call returns. */
 int nbos_snapshot_create_host(const nbos_snapshot_desc *desc, void *cuda_stream,
                               nbos_snapshot **out);
+
+/*
+ * Refresh an existing snapshot from new cluster state of the same shape (same N, H, R, key order
+ * and flags as at creation; `desc` carries the new arrays and limits): the per-host records of
+ * Sections 3.2.1 / 3.4.1 are derived again with the key widths, packing layout and visiting-order
+ * machinery chosen at creation. Unlike creation this reads nothing back and never synchronises:
+ * it only queues work on `cuda_stream`, so a scheduler tick can queue "update, place, update,
+ * place ..." without waiting. The price is that problems are reported late: if the new state
+ * has a value outside the supported range, or does not fit the stored layout (more idle GPUs,
+ * a larger subscription or capacity than the widths allow, a GPU count per host the snapshot did
+ * not have), the device status word is raised, the tables and every placement made from them are
+ * undefined, and nbos_snapshot_status returns NBOS_ERR_RANGE / NBOS_ERR_STALE_LAYOUT; destroy the
+ * snapshot and create a new one then. A successful update also clears an earlier status.
+ * The caller must make sure that no placement on ANOTHER stream is still using the snapshot;
+ * work queued earlier on the same stream is ordered before the update.
+ *   nbos_snapshot_update       arrays are DEVICE memory (16-byte aligned), read by the queued work
+ *   nbos_snapshot_update_host  arrays are HOST memory; staged through the library's memory pool
+ * Errors at call time: INVALID_ARG (shape / flags differ, NULL or misaligned pointers, bad limit),
+ * NO_MEMORY, CUDA.
+ */
+int nbos_snapshot_update(nbos_snapshot *snap, const nbos_snapshot_desc *desc, void *cuda_stream);
+int nbos_snapshot_update_host(nbos_snapshot *snap, const nbos_snapshot_desc *desc, void *cuda_stream);
 
 /* Frees the handle (and what nbos_snapshot_create_host allocated). The caller must make sure no
  * nbos_place_batch on this snapshot is still running. NULL is accepted. */
@@ -339,7 +363,8 @@ int nbos_scale_out_deficit(const int32_t *found, int32_t n_snapshots, int64_t ba
 
 /* Synchronises `cuda_stream` and returns the sticky device status of this snapshot: NBOS_OK, or
  * NBOS_ERR_DEVICE_TIMEOUT if some kernel gave up on a bounded wait (its outputs are then
- * undefined). */
+ * undefined), NBOS_ERR_RANGE / NBOS_ERR_STALE_LAYOUT after an nbos_snapshot_update whose new state
+ * was invalid / did not fit the snapshot's layout. */
 int nbos_snapshot_status(const nbos_snapshot *snap, void *cuda_stream);
 
 const char *nbos_strerror(int status);

@@ -22,6 +22,7 @@ NBOS_ERR_CUDA = -3
 NBOS_ERR_UNSUPPORTED_DEVICE = -4
 NBOS_ERR_DEVICE_TIMEOUT = -5
 NBOS_ERR_NO_MEMORY = -6
+NBOS_ERR_STALE_LAYOUT = -7
 
 NBOS_KEY_IDLE_FIRST = 0
 NBOS_KEY_SR_FIRST = 1
@@ -37,6 +38,7 @@ NBOS_PROBE_MIX_BOTH = 2
 # every symbol include/nbos.h and include/nbos_probe.h declare
 EXPORTED_SYMBOLS = (
     "nbos_snapshot_workspace_bytes", "nbos_snapshot_create", "nbos_snapshot_create_host",
+    "nbos_snapshot_update", "nbos_snapshot_update_host",
     "nbos_snapshot_destroy", "nbos_snapshot_get_info", "nbos_place_batch", "nbos_place_batch_ex",
     "nbos_place_batch_host", "nbos_place_batch_noalloc", "nbos_select_executors",
     "nbos_cluster_sums", "nbos_scale_out_deficit", "nbos_place_batch_sequential",
@@ -113,6 +115,8 @@ def load_library() -> ctypes.CDLL:
     lib.nbos_snapshot_workspace_bytes.argtypes = [P(nbos_snapshot_desc), P(sz)]
     lib.nbos_snapshot_create.argtypes = [P(nbos_snapshot_desc), vp, sz, vp, P(vp)]
     lib.nbos_snapshot_create_host.argtypes = [P(nbos_snapshot_desc), vp, P(vp)]
+    lib.nbos_snapshot_update.argtypes = [vp, P(nbos_snapshot_desc), vp]
+    lib.nbos_snapshot_update_host.argtypes = [vp, P(nbos_snapshot_desc), vp]
     lib.nbos_snapshot_destroy.argtypes = [vp]
     lib.nbos_snapshot_get_info.argtypes = [vp, P(nbos_snapshot_info)]
     lib.nbos_place_batch.argtypes = [vp, vp, i64, vp, vp, vp]
@@ -244,6 +248,30 @@ def nbos_snapshot_create_host(n_snapshots, n_hosts, limit_num, limit_den, gpus_t
     out = ctypes.c_void_p(0)
     _check(lib.nbos_snapshot_create_host(ctypes.byref(d), _stream_ptr(stream), ctypes.byref(out)))
     return Snapshot(int(out.value), n_snapshots, n_hosts)
+
+
+def _update(fn_name, device_type, snap, limit_num, limit_den, arrays, stream):
+    info = nbos_snapshot_get_info(snap)
+    d, keep = _make_desc(snap.n_snapshots, snap.n_hosts, info.replicas_R, info.key_order, info.flags,
+                         limit_num, limit_den, arrays, device_type)
+    _check(getattr(load_library(), fn_name)(snap.handle, ctypes.byref(d), _stream_ptr(stream)))
+    if device_type == "cuda":
+        snap.keep = snap.keep[:1] + keep   # the queued kernels read the new arrays: keep them alive
+
+
+def nbos_snapshot_update(snap: Snapshot, limit_num, limit_den, gpus_total, gpus_subscribed,
+                         gpus_committed, vram_gb, millicpus, mem_mb, stream=None) -> None:
+    """Refresh the snapshot from new device arrays of the same shape; asynchronous, no read-back.
+    Problems with the new state show up in nbos_snapshot_status."""
+    _update("nbos_snapshot_update", "cuda", snap, limit_num, limit_den,
+            (gpus_total, gpus_subscribed, gpus_committed, vram_gb, millicpus, mem_mb), stream)
+
+
+def nbos_snapshot_update_host(snap: Snapshot, limit_num, limit_den, gpus_total, gpus_subscribed,
+                              gpus_committed, vram_gb, millicpus, mem_mb, stream=None) -> None:
+    """Same from host (CPU tensor) arrays."""
+    _update("nbos_snapshot_update_host", "cpu", snap, limit_num, limit_den,
+            (gpus_total, gpus_subscribed, gpus_committed, vram_gb, millicpus, mem_mb), stream)
 
 
 def nbos_snapshot_destroy(snap: Snapshot) -> None:

@@ -242,6 +242,61 @@ int nbos_snapshot_create_host(const nbos_snapshot_desc *desc, void *cuda_stream,
     return NBOS_OK;
 }
 
+static int check_update_desc(const nbos_snapshot *snap, const nbos_snapshot_desc *desc)
+{
+    if (!snap) return fail(NBOS_ERR_INVALID_ARG, "snapshot is NULL");
+    int rc = check_desc_full(desc);
+    if (rc) return rc;
+    if (desc->n_snapshots != snap->N || desc->n_hosts != snap->H || desc->replicas_R != snap->R ||
+        desc->key_order != snap->key_order || desc->flags != snap->flags)
+        return fail(NBOS_ERR_INVALID_ARG, "update: shape, R, key order and flags must be those the snapshot was created with");
+    int device = -1;
+    NBOS_CUDA_TRY(cudaGetDevice(&device));
+    if (device != snap->device) return fail(NBOS_ERR_INVALID_ARG, "update: the snapshot belongs to device %d", snap->device);
+    return NBOS_OK;
+}
+
+int nbos_snapshot_update(nbos_snapshot *snap, const nbos_snapshot_desc *desc, void *cuda_stream)
+{
+    int rc = check_update_desc(snap, desc);
+    if (rc) return rc;
+    const void *arrays[6] = {desc->gpus_total, desc->gpus_subscribed, desc->gpus_committed,
+                             desc->vram_gb, desc->millicpus, desc->mem_mb};
+    for (int i = 0; i < 6; ++i)
+        if (!aligned(arrays[i], 16)) return fail(NBOS_ERR_INVALID_ARG, "host-state array %d is not 16-byte aligned", i);
+    return update_snapshot(snap, desc, desc->gpus_total, desc->gpus_subscribed, desc->gpus_committed,
+                           desc->vram_gb, desc->millicpus, desc->mem_mb, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int nbos_snapshot_update_host(nbos_snapshot *snap, const nbos_snapshot_desc *desc, void *cuda_stream)
+{
+    int rc = check_update_desc(snap, desc);
+    if (rc) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    HostPipe *pipe = nullptr;
+    rc = host_pipe(snap->device, &pipe);
+    if (rc) return rc;
+    const size_t cells = (size_t)snap->N * snap->H;
+    const size_t arr_bytes = (cells * sizeof(int32_t) + 255) & ~(size_t)255;
+    void *staging = nullptr;
+    cudaError_t e = cudaMallocFromPoolAsync(&staging, 6 * arr_bytes, pipe->pool, stream);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(NBOS_ERR_NO_MEMORY, "device allocation failed: %s", cudaGetErrorString(e));
+    }
+    const int32_t *src[6] = {desc->gpus_total, desc->gpus_subscribed, desc->gpus_committed,
+                             desc->vram_gb, desc->millicpus, desc->mem_mb};
+    const int32_t *dev[6];
+    for (int i = 0; i < 6 && e == cudaSuccess; ++i) {
+        dev[i] = reinterpret_cast<const int32_t *>(static_cast<char *>(staging) + i * arr_bytes);
+        e = cudaMemcpyAsync(const_cast<int32_t *>(dev[i]), src[i], cells * sizeof(int32_t), cudaMemcpyHostToDevice, stream);
+    }
+    rc = e == cudaSuccess ? update_snapshot(snap, desc, dev[0], dev[1], dev[2], dev[3], dev[4], dev[5], stream)
+                          : cuda_fail(e, "copying host-state arrays to the device");
+    cudaFreeAsync(staging, stream);
+    return rc;
+}
+
 int nbos_snapshot_destroy(nbos_snapshot *snap)
 {
     if (!snap) return NBOS_OK;
@@ -416,7 +471,10 @@ int nbos_snapshot_status(const nbos_snapshot *snap, void *cuda_stream)
     unsigned int word = 0;
     NBOS_CUDA_TRY(cudaMemcpyAsync(&word, snap->d_status, sizeof(word), cudaMemcpyDeviceToHost, stream));
     NBOS_CUDA_TRY(cudaStreamSynchronize(stream));
-    if (word) return fail(NBOS_ERR_DEVICE_TIMEOUT, "a kernel gave up on a bounded wait (status word 0x%x)", word);
+    if (word & STATUS_WAIT_TIMEOUT) return fail(NBOS_ERR_DEVICE_TIMEOUT, "a kernel gave up on a bounded wait (status word 0x%x)", word);
+    if (word & STATUS_BAD_VALUES) return fail(NBOS_ERR_RANGE, "the last update brought a value outside the supported range (status word 0x%x)", word);
+    if (word & STATUS_STALE_LAYOUT) return fail(NBOS_ERR_STALE_LAYOUT, "the last update does not fit the snapshot's layout (status word 0x%x)", word);
+    if (word) return fail(NBOS_ERR_CUDA, "unknown status word 0x%x", word);
     return NBOS_OK;
 }
 
@@ -430,6 +488,7 @@ const char *nbos_strerror(int status)
         case NBOS_ERR_UNSUPPORTED_DEVICE: return "unsupported device (needs compute capability 10.x)";
         case NBOS_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
         case NBOS_ERR_NO_MEMORY: return "out of memory or workspace too small";
+        case NBOS_ERR_STALE_LAYOUT: return "updated state does not fit the snapshot's layout";
     }
     return "unknown status";
 }

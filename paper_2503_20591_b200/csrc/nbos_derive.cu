@@ -21,6 +21,13 @@ struct ScanArgs {
     longlong2 limit0;         // used instead of limits[0] when `limits` is null (single snapshot)
     SnapStats *stats;
     int H, R, flags;
+    // update mode (null status = create mode): the new state must fit the layout chosen when the
+    // snapshot was created; a host that does not raises STATUS_STALE_LAYOUT in the status word
+    unsigned int *status;
+    const long long *lambda;   // per snapshot; null = static key
+    const int *g_single;       // per snapshot: the one GPU count of a static-key snapshot (0 = none)
+    unsigned long long sr_field_max;
+    int idle_max, pack_enabled, fmax[4];
 };
 
 // `num_r` is the limit's numerator times R (R already cancelled for the dynamic limit).
@@ -74,6 +81,18 @@ __global__ void limits_from_sums_kernel(const unsigned long long *sums, longlong
     if (n < N) limits[n] = make_longlong2((long long)sums[(size_t)n * 4 + 1], (long long)sums[(size_t)n * 4 + 0]);
 }
 
+// Per-snapshot values travel to the device inside kernel arguments (captured at launch, so no
+// host buffer has to outlive the call and no stream synchronisation is implied).
+struct LimitChunk {
+    longlong2 v[128];
+    int first, count;
+};
+__global__ void set_limits_kernel(longlong2 *limits, const LimitChunk c)
+{
+    const int i = threadIdx.x;
+    if (i < c.count) limits[c.first + i] = c.v[i];
+}
+
 // Auto-scaler rule (Section 3.4.2) next to the sums: sums[n*4+3] = +1 if sum G < f * sum C (scale
 // out), -1 if f * sum C < sum G (servers may be released), 0 if equal; f = f_num / f_den.
 __global__ void autoscale_kernel(unsigned long long *sums, int N, long long f_num, long long f_den)
@@ -109,6 +128,7 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
     int idle_max = 0, g_min_inv = 0;  // INT_MAX - smallest G seen, 0 = none
     unsigned long long sub_max = 0ull;
     int max_gcap1 = 0, max_av = 0, max_ac = 0, max_am = 0;  // max_gcap1 = largest gmax + 1
+    unsigned int upd = 0u;
     for (int h = blockIdx.x * blockDim.x + threadIdx.x; h < a.H; h += gridDim.x * blockDim.x) {
         const size_t i = (size_t)n * a.H + h;
         const int G = a.G[i], S = a.S[i], C = a.C[i];
@@ -133,6 +153,30 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
         max_av = max(max_av, a.AV[i]);
         max_ac = max(max_ac, a.AC[i]);
         max_am = max(max_am, a.AM[i]);
+        if (a.status) {
+            bool stale = G - C > a.idle_max;
+            long long w = 1;
+            if (G >= 1) {
+                if (a.lambda) {
+                    const long long lam = a.lambda[n];
+                    if (lam % G) stale = true; else w = lam / G;
+                } else if (G != a.g_single[n]) {
+                    stale = true;
+                }
+            }
+            if (gm >= 0) {
+                unsigned long long top = (unsigned long long)S + (unsigned long long)gm;
+                if (a.flags & NBOS_ROOM_FOR_COMMITS) top = max(top, (unsigned long long)((lim.x * (long long)G) / lim.y));
+                if (top > a.sr_field_max / (unsigned long long)w) stale = true;
+            }
+            if (a.pack_enabled && (gm > a.fmax[0] || a.AV[i] > a.fmax[1] || a.AC[i] > a.fmax[2] || a.AM[i] > a.fmax[3]))
+                stale = true;
+            if (stale) upd |= STATUS_STALE_LAYOUT;
+        }
+    }
+    if (a.status) {
+        if (err) upd |= STATUS_BAD_VALUES;
+        if (upd) atomicOr(a.status, upd);
     }
     if (err) atomicOr(&s_err, err);
     atomicMax(&s_idle_max, idle_max);
@@ -309,8 +353,9 @@ Layout workspace_layout(int N, int Hpad)
     l.off_status = o;  o = up(o + 256);
     l.off_limits = o;  o = up(o + (size_t)N * sizeof(longlong2));
     l.off_sums = o;    o = up(o + (size_t)N * 4 * sizeof(unsigned long long));
-    l.off_lambda = o;  o = up(o + (size_t)N * sizeof(long long));
     l.off_stats = o;   o = up(o + (size_t)N * sizeof(SnapStats));
+    l.off_lambda = o;  o = up(o + (size_t)N * sizeof(long long));
+    l.off_g_single = o; o = up(o + (size_t)N * sizeof(int));
     l.off_feas = o;    o = up(o + (size_t)N * Hpad * sizeof(int4));
     l.off_ab = o;      o = up(o + (size_t)N * Hpad * sizeof(ulonglong2));
     l.off_pk = o;      o = up(o + (size_t)N * Hpad * sizeof(uint4));
@@ -336,49 +381,128 @@ int launch_cluster_sums(const int32_t *d_G, const int32_t *d_S, const int32_t *d
     return NBOS_OK;
 }
 
+namespace {
+
+struct DeriveCtx {
+    nbos_snapshot *s;
+    const int32_t *G, *S, *C, *AV, *AC, *AM;
+    cudaStream_t stream;
+    Layout lay;
+    char *ws;
+    longlong2 *d_limits;
+    const longlong2 *limits_arg;
+    longlong2 limit0;
+    int bx;
+};
+
+// Clear the per-derivation state and put the limits on the device (or compute them there).
+int stage_limits(DeriveCtx &c, const nbos_snapshot_desc *d)
+{
+    nbos_snapshot *s = c.s;
+    const int N = s->N, H = s->H;
+    const bool dynamic_limit = (s->flags & NBOS_LIMIT_CLUSTER_SR) != 0;
+    // status word, limits, sums and scan statistics are contiguous: one clear (lambda and g_single,
+    // which an update keeps, lie behind them)
+    NBOS_CUDA_TRY(cudaMemsetAsync(c.ws + c.lay.off_status, 0, c.lay.off_lambda - c.lay.off_status, c.stream));
+    c.limits_arg = c.d_limits;
+    c.limit0 = make_longlong2(0, 1);
+    if (dynamic_limit) {
+        unsigned long long *d_sums = reinterpret_cast<unsigned long long *>(c.ws + c.lay.off_sums);
+        sums_kernel<<<dim3(c.bx, N), 256, 0, c.stream>>>(c.G, c.S, c.C, H, d_sums);
+        limits_from_sums_kernel<<<(N + 255) / 256, 256, 0, c.stream>>>(d_sums, c.d_limits, N);
+    } else if (N == 1) {
+        // a single snapshot's fixed limit travels in the kernel arguments
+        c.limits_arg = nullptr;
+        c.limit0 = make_longlong2((long long)d->limit_num[0] * s->R, d->limit_den[0]);
+    } else {
+        for (int first = 0; first < N; first += 128) {
+            LimitChunk chunk;
+            chunk.first = first;
+            chunk.count = N - first < 128 ? N - first : 128;
+            for (int i = 0; i < chunk.count; ++i)
+                chunk.v[i] = make_longlong2((long long)d->limit_num[first + i] * s->R, d->limit_den[first + i]);
+            set_limits_kernel<<<1, 128, 0, c.stream>>>(c.d_limits, chunk);
+        }
+    }
+    NBOS_CUDA_TRY(cudaGetLastError());
+    return NBOS_OK;
+}
+
+// emit -> rank -> finalize with the layout stored in the handle
+int emit_tables(DeriveCtx &c)
+{
+    nbos_snapshot *s = c.s;
+    const int N = s->N, H = s->H, Hpad = s->Hpad;
+    const KeyLayout &k = s->key;
+    long long *d_lambda = reinterpret_cast<long long *>(c.ws + c.lay.off_lambda);
+    int4 *tmp_feas = reinterpret_cast<int4 *>(c.ws + c.lay.off_tmp_feas);
+    void *tmp_ab = c.ws + c.lay.off_tmp_ab;
+    unsigned long long *sortkey = reinterpret_cast<unsigned long long *>(c.ws + c.lay.off_sortkey);
+    unsigned int *perm = reinterpret_cast<unsigned int *>(c.ws + c.lay.off_perm);
+    int4 *tmp_seq = reinterpret_cast<int4 *>(c.ws + c.lay.off_tmp_seq);
+    EmitArgs ea{c.G, c.S, c.C, c.AV, c.AC, c.AM, c.limits_arg, c.limit0, k.static_key ? nullptr : d_lambda,
+                s->presorted ? perm : nullptr, tmp_feas, tmp_seq, tmp_ab, sortkey,
+                H, Hpad, s->R, s->flags, s->key_order, s->idle_max, k.bits_idle, k.bits_sr, k.bits_id};
+    dim3 grid((Hpad + 255) / 256, N);
+    if (k.key_bits == 32)
+        emit_kernel<unsigned int, uint2><<<grid, 256, 0, c.stream>>>(ea);
+    else
+        emit_kernel<unsigned long long, ulonglong2><<<grid, 256, 0, c.stream>>>(ea);
+    if (s->presorted)
+        rank_kernel<<<dim3((Hpad + 255) / 256, (Hpad + kRankChunk - 1) / kRankChunk, N), 256, 0, c.stream>>>(sortkey, perm, Hpad);
+    FinalizeArgs fa{tmp_feas, tmp_ab, s->presorted ? perm : nullptr, reinterpret_cast<int4 *>(c.ws + c.lay.off_feas),
+                    c.ws + c.lay.off_ab, reinterpret_cast<uint4 *>(c.ws + c.lay.off_pk), Hpad, s->pack};
+    if (k.key_bits == 32)
+        finalize_kernel<uint2><<<grid, 256, 0, c.stream>>>(fa);
+    else
+        finalize_kernel<ulonglong2><<<grid, 256, 0, c.stream>>>(fa);
+    NBOS_CUDA_TRY(cudaGetLastError());
+    return NBOS_OK;
+}
+
+DeriveCtx make_ctx(nbos_snapshot *s, const int32_t *d_G, const int32_t *d_S, const int32_t *d_C,
+                   const int32_t *d_AV, const int32_t *d_AC, const int32_t *d_AM, cudaStream_t stream)
+{
+    DeriveCtx c;
+    c.s = s;
+    c.G = d_G; c.S = d_S; c.C = d_C; c.AV = d_AV; c.AC = d_AC; c.AM = d_AM;
+    c.stream = stream;
+    c.lay = workspace_layout(s->N, s->Hpad);
+    c.ws = static_cast<char *>(s->workspace);
+    c.d_limits = reinterpret_cast<longlong2 *>(c.ws + c.lay.off_limits);
+    c.limits_arg = c.d_limits;
+    c.limit0 = make_longlong2(0, 1);
+    c.bx = (s->H + 255) / 256;
+    if (c.bx > 64) c.bx = 64;
+    return c;
+}
+
+}  // namespace
+
 int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t *d_G,
                     const int32_t *d_S, const int32_t *d_C, const int32_t *d_AV,
                     const int32_t *d_AC, const int32_t *d_AM, cudaStream_t stream)
 {
     const int N = s->N, H = s->H, Hpad = s->Hpad;
-    const Layout lay = workspace_layout(N, Hpad);
-    char *ws = static_cast<char *>(s->workspace);
-    longlong2 *d_limits = reinterpret_cast<longlong2 *>(ws + lay.off_limits);
-    unsigned long long *d_sums = reinterpret_cast<unsigned long long *>(ws + lay.off_sums);
-    const bool dynamic_limit = (s->flags & NBOS_LIMIT_CLUSTER_SR) != 0;
-    long long *d_lambda = reinterpret_cast<long long *>(ws + lay.off_lambda);
-    SnapStats *d_stats = reinterpret_cast<SnapStats *>(ws + lay.off_stats);
+    DeriveCtx c = make_ctx(s, d_G, d_S, d_C, d_AV, d_AC, d_AM, stream);
+    long long *d_lambda = reinterpret_cast<long long *>(c.ws + c.lay.off_lambda);
+    int *d_g_single = reinterpret_cast<int *>(c.ws + c.lay.off_g_single);
+    SnapStats *d_stats = reinterpret_cast<SnapStats *>(c.ws + c.lay.off_stats);
 
-    // limits -> device
-    longlong2 *h_limits = static_cast<longlong2 *>(malloc(sizeof(longlong2) * (size_t)N));
     SnapStats *h_stats = static_cast<SnapStats *>(malloc(sizeof(SnapStats) * (size_t)N));
     long long *h_lambda = static_cast<long long *>(malloc(sizeof(long long) * (size_t)N));
+    int *h_g_single = static_cast<int *>(malloc(sizeof(int) * (size_t)N));
     struct Free {
         void *a, *b, *c;
         ~Free() { free(a); free(b); free(c); }
-    } guard{h_limits, h_stats, h_lambda};
-    if (!h_limits || !h_stats || !h_lambda) return fail(NBOS_ERR_NO_MEMORY, "host allocation failed");
-    if (!dynamic_limit)
-        for (int n = 0; n < N; ++n) h_limits[n] = make_longlong2((long long)d->limit_num[n] * s->R, d->limit_den[n]);
+    } guard{h_stats, h_lambda, h_g_single};
+    if (!h_stats || !h_lambda || !h_g_single) return fail(NBOS_ERR_NO_MEMORY, "host allocation failed");
 
-    // status word, limits, lambda and scan statistics are contiguous: one clear
-    NBOS_CUDA_TRY(cudaMemsetAsync(ws + lay.off_status, 0, lay.off_feas - lay.off_status, stream));
-    int bx = (H + 255) / 256;
-    if (bx > 64) bx = 64;
-    if (dynamic_limit) {
-        sums_kernel<<<dim3(bx, N), 256, 0, stream>>>(d_G, d_S, d_C, H, d_sums);
-        limits_from_sums_kernel<<<(N + 255) / 256, 256, 0, stream>>>(d_sums, d_limits, N);
-        NBOS_CUDA_TRY(cudaGetLastError());
-    } else if (N > 1) {
-        NBOS_CUDA_TRY(cudaMemcpyAsync(d_limits, h_limits, sizeof(longlong2) * (size_t)N,
-                                      cudaMemcpyHostToDevice, stream));
-    }
-    // a single snapshot's fixed limit travels in the kernel arguments instead of a copy
-    const longlong2 *limits_arg = (N == 1 && !dynamic_limit) ? nullptr : d_limits;
-    const longlong2 limit0 = (N == 1 && !dynamic_limit) ? h_limits[0] : make_longlong2(0, 1);
-
-    ScanArgs sa{d_G, d_S, d_C, d_AV, d_AC, d_AM, limits_arg, limit0, d_stats, H, s->R, s->flags};
-    scan_kernel<<<dim3(bx, N), 256, 0, stream>>>(sa);
+    int rc = stage_limits(c, d);
+    if (rc) return rc;
+    ScanArgs sa{d_G, d_S, d_C, d_AV, d_AC, d_AM, c.limits_arg, c.limit0, d_stats, H, s->R, s->flags,
+                nullptr, nullptr, nullptr, 0ull, 0, 0, {0, 0, 0, 0}};
+    scan_kernel<<<dim3(c.bx, N), 256, 0, stream>>>(sa);
     NBOS_CUDA_TRY(cudaGetLastError());
     NBOS_CUDA_TRY(cudaMemcpyAsync(h_stats, d_stats, sizeof(SnapStats) * (size_t)N,
                                   cudaMemcpyDeviceToHost, stream));
@@ -395,13 +519,17 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
         if (st.err & ERR_G_TOO_LARGE)
             return fail(NBOS_ERR_RANGE, "snapshot %d: more than %d GPUs on some host", n, NBOS_MAX_GPUS_PER_HOST);
         unsigned long long lambda = 1;
+        int distinct = 0, single = 0;
         for (int G = 1; G <= NBOS_MAX_GPUS_PER_HOST; ++G) {
             if (!(st.g_mask[G >> 6] >> (G & 63) & 1ull)) continue;
+            ++distinct;
+            single = G;
             lambda = lambda / gcd_u64(lambda, (unsigned long long)G) * (unsigned long long)G;
             if (lambda > (1ull << 40))
                 return fail(NBOS_ERR_RANGE, "snapshot %d: GPU counts per host too diverse for an exact 63-bit key", n);
         }
         h_lambda[n] = (long long)lambda;
+        h_g_single[n] = distinct == 1 ? single : 0;
         if (st.idle_max > idle_max) idle_max = st.idle_max;
         if (st.g_min_inv != 0) {
             const unsigned long long w_max = lambda / (unsigned long long)(INT_MAX - st.g_min_inv);
@@ -431,13 +559,17 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
         if (st.max_am > fmax[3]) fmax[3] = st.max_am;
     }
     s->key = k;
+    // the idle field can hold up to 2^bits - 1: use all of it, so that a later update may bring
+    // hosts with more idle GPUs than any host has now
+    idle_max = (int)((1u << k.bits_idle) - 1u);
+    s->idle_max = idle_max;
 
     // packed capacity test: the two widest components become the high fields of the two words
     PackLayout pk = {};
     if (k.key_bits == 32) {
         int width[4], order[4] = {0, 1, 2, 3};
         width[0] = bits_for((unsigned long long)fmax[0] + 2);  // stored +1, and one more for "fits nowhere"
-        for (int c = 1; c < 4; ++c) width[c] = fmax[c] ? bits_for((unsigned long long)fmax[c]) : 1;
+        for (int c2 = 1; c2 < 4; ++c2) width[c2] = fmax[c2] ? bits_for((unsigned long long)fmax[c2]) : 1;
         for (int i = 0; i < 4; ++i)
             for (int j = i + 1; j < 4; ++j)
                 if (width[order[j]] > width[order[i]]) { int t = order[i]; order[i] = order[j]; order[j] = t; }
@@ -450,7 +582,10 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
             pk.enabled = 1;
             pk.guards = 0x80000000u | (1u << lo_a);
             pk.guards1 = 0x80000000u | (1u << lo_b);
-            for (int c = 0; c < 4; ++c) pk.fmax[c] = fmax[c];
+            // largest value each field can take (not merely the largest present now): asks up to it
+            // are compared exactly, and a later update may raise capacities up to it
+            pk.fmax[0] = (int)((1u << width[0]) - 3u);
+            for (int c2 = 1; c2 < 4; ++c2) pk.fmax[c2] = (int)((1u << width[c2]) - 1u);
             pk.fword[order[0]] = 0; pk.fshift[order[0]] = lo_a + 1;
             pk.fword[order[3]] = 0; pk.fshift[order[3]] = 0;
             pk.fword[order[1]] = 1; pk.fshift[order[1]] = lo_b + 1;
@@ -458,46 +593,45 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
         }
     }
     s->pack = pk;
-
-    if (!k.static_key)
-        NBOS_CUDA_TRY(cudaMemcpyAsync(d_lambda, h_lambda, sizeof(long long) * (size_t)N,
-                                      cudaMemcpyHostToDevice, stream));
     s->presorted = Hpad <= kSortMaxHosts;
-    int4 *tmp_feas = reinterpret_cast<int4 *>(ws + lay.off_tmp_feas);
-    void *tmp_ab = ws + lay.off_tmp_ab;
-    unsigned long long *sortkey = reinterpret_cast<unsigned long long *>(ws + lay.off_sortkey);
-    unsigned int *perm = reinterpret_cast<unsigned int *>(ws + lay.off_perm);
-    int4 *tmp_seq = reinterpret_cast<int4 *>(ws + lay.off_tmp_seq);
-    EmitArgs ea{d_G, d_S, d_C, d_AV, d_AC, d_AM, limits_arg, limit0, k.static_key ? nullptr : d_lambda,
-                s->presorted ? perm : nullptr, tmp_feas, tmp_seq, tmp_ab, sortkey,
-                H, Hpad, s->R, s->flags, s->key_order, idle_max, k.bits_idle, k.bits_sr, k.bits_id};
-    dim3 grid((Hpad + 255) / 256, N);
-    if (k.key_bits == 32)
-        emit_kernel<unsigned int, uint2><<<grid, 256, 0, stream>>>(ea);
-    else
-        emit_kernel<unsigned long long, ulonglong2><<<grid, 256, 0, stream>>>(ea);
-    NBOS_CUDA_TRY(cudaGetLastError());
 
-    // visiting order
-    if (s->presorted) {
-        rank_kernel<<<dim3((Hpad + 255) / 256, (Hpad + kRankChunk - 1) / kRankChunk, N), 256, 0, stream>>>(sortkey, perm, Hpad);
-        NBOS_CUDA_TRY(cudaGetLastError());
-    }
-    FinalizeArgs fa{tmp_feas, tmp_ab, s->presorted ? perm : nullptr, reinterpret_cast<int4 *>(ws + lay.off_feas), ws + lay.off_ab,
-                    reinterpret_cast<uint4 *>(ws + lay.off_pk), Hpad, pk};
-    if (k.key_bits == 32)
-        finalize_kernel<uint2><<<grid, 256, 0, stream>>>(fa);
-    else
-        finalize_kernel<ulonglong2><<<grid, 256, 0, stream>>>(fa);
-    NBOS_CUDA_TRY(cudaGetLastError());
-    s->d_status = reinterpret_cast<unsigned int *>(ws + lay.off_status);
-    s->d_feas = reinterpret_cast<const int4 *>(ws + lay.off_feas);
-    s->d_ab = ws + lay.off_ab;
-    s->d_pk = reinterpret_cast<const uint4 *>(ws + lay.off_pk);
-    s->d_host_feas = tmp_feas;
-    s->d_host_ab = tmp_ab;
-    s->d_host_seq = tmp_seq;
+    // what a later nbos_snapshot_update checks the new state against
+    if (!k.static_key)
+        NBOS_CUDA_TRY(cudaMemcpyAsync(d_lambda, h_lambda, sizeof(long long) * (size_t)N, cudaMemcpyHostToDevice, stream));
+    NBOS_CUDA_TRY(cudaMemcpyAsync(d_g_single, h_g_single, sizeof(int) * (size_t)N, cudaMemcpyHostToDevice, stream));
+
+    rc = emit_tables(c);
+    if (rc) return rc;
+    s->d_status = reinterpret_cast<unsigned int *>(c.ws + c.lay.off_status);
+    s->d_feas = reinterpret_cast<const int4 *>(c.ws + c.lay.off_feas);
+    s->d_ab = c.ws + c.lay.off_ab;
+    s->d_pk = reinterpret_cast<const uint4 *>(c.ws + c.lay.off_pk);
+    s->d_host_feas = reinterpret_cast<const int4 *>(c.ws + c.lay.off_tmp_feas);
+    s->d_host_ab = c.ws + c.lay.off_tmp_ab;
+    s->d_host_seq = reinterpret_cast<const int4 *>(c.ws + c.lay.off_tmp_seq);
     return NBOS_OK;
+}
+
+// Re-derive the tables of an existing snapshot from new state, keeping the key and packing layout
+// chosen at creation. Nothing is read back: a state that does not fit the layout is reported
+// through the status word.
+int update_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t *d_G,
+                    const int32_t *d_S, const int32_t *d_C, const int32_t *d_AV,
+                    const int32_t *d_AC, const int32_t *d_AM, cudaStream_t stream)
+{
+    DeriveCtx c = make_ctx(s, d_G, d_S, d_C, d_AV, d_AC, d_AM, stream);
+    int rc = stage_limits(c, d);
+    if (rc) return rc;
+    ScanArgs sa{d_G, d_S, d_C, d_AV, d_AC, d_AM, c.limits_arg, c.limit0,
+                reinterpret_cast<SnapStats *>(c.ws + c.lay.off_stats), s->H, s->R, s->flags,
+                s->d_status,
+                s->key.static_key ? nullptr : reinterpret_cast<const long long *>(c.ws + c.lay.off_lambda),
+                reinterpret_cast<const int *>(c.ws + c.lay.off_g_single),
+                s->key.bits_sr >= 64 ? ~0ull : ((1ull << s->key.bits_sr) - 1ull), s->idle_max, s->pack.enabled,
+                {s->pack.fmax[0], s->pack.fmax[1], s->pack.fmax[2], s->pack.fmax[3]}};
+    scan_kernel<<<dim3(c.bx, s->N), 256, 0, stream>>>(sa);
+    NBOS_CUDA_TRY(cudaGetLastError());
+    return emit_tables(c);
 }
 
 }  // namespace nbos

@@ -30,6 +30,11 @@ struct SnapStats {                 // one per snapshot, filled by the scan kerne
     int max_gcap1, max_av, max_ac, max_am;  // maxima of gmax + 1 and of the three capacities
     unsigned long long g_mask[16]; // bit G set if some host has G GPUs (G in 1..1023)
 };
+enum : unsigned int {  // bits of the snapshot's device status word
+    STATUS_WAIT_TIMEOUT = 1u,   // a kernel gave up on a bounded wait
+    STATUS_STALE_LAYOUT = 2u,   // nbos_snapshot_update: the new state does not fit the stored layout
+    STATUS_BAD_VALUES = 4u,     // nbos_snapshot_update: a value outside the supported range
+};
 enum : unsigned int {
     ERR_NEGATIVE = 1u,        // some value < 0
     ERR_COMMITTED_GT_TOTAL = 2u,
@@ -37,7 +42,7 @@ enum : unsigned int {
 };
 
 struct Layout {
-    size_t off_status, off_limits, off_sums, off_lambda, off_stats, off_feas, off_ab, off_pk;
+    size_t off_status, off_limits, off_sums, off_stats, off_lambda, off_g_single, off_feas, off_ab, off_pk;
     size_t off_tmp_feas, off_tmp_ab, off_tmp_seq, off_sortkey, off_perm, total;
 };
 Layout workspace_layout(int n_snapshots, int hosts_padded);
@@ -78,6 +83,7 @@ struct nbos_snapshot {
     const uint4 *d_pk;    // [N][Hpad] (word0, word1, A, B), only when pack.enabled
     nbos::PackLayout pack;
     int presorted;
+    int idle_max;             // the key's idle field stores idle_max - (G - C)
     // the same records in host-index order (what the derivation staged), for sequential placement
     const int4 *d_host_feas;
     const void *d_host_ab;
@@ -96,6 +102,10 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *host_desc, const
 // Cluster sums + auto-scaler sign per snapshot into d_out [N][4] (nbos_derive.cu).
 int launch_cluster_sums(const int32_t *d_G, const int32_t *d_S, const int32_t *d_C, int N, int H,
                         long long f_num, long long f_den, long long *d_out, cudaStream_t stream);
+
+int update_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *host_desc, const int32_t *d_G,
+                    const int32_t *d_S, const int32_t *d_C, const int32_t *d_AV,
+                    const int32_t *d_AC, const int32_t *d_AM, cudaStream_t stream);
 
 // a1-a9: the placement launch (nbos_place.cu). The pointers are those of the whole batch; the
 // launch handles the flattened requests [range_first, range_first + range_count) of the N * batch
