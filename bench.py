@@ -50,6 +50,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--cpu-sample", type=int, default=None, help="requests in the CPU sample")
+    ap.add_argument("--fresh-snapshot", action="store_true",
+                    help="create a new snapshot in every step instead of refreshing one")
     ap.add_argument("--all-workloads", action="store_true",
                     help="also time the placement kernel on all five benchmark shapes")
     ap.add_argument("--lanes", type=int, default=0,
@@ -218,9 +220,20 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
     launch_cfg = nb.launch_config(lanes_per_request=args.lanes) if args.lanes else None
 
+    # The snapshot object is created once; every step refreshes it from the cluster-state arrays
+    # (all derivation kernels run again, nothing is read back) and places one batch. With
+    # --fresh-snapshot every step creates a new snapshot instead (one host synchronisation each).
+    live = None if args.fresh_snapshot else nb.nbos_snapshot_create(
+        w.n_snapshots, w.n_hosts, lim_num, lim_den, *d_state, replicas_R=w.replicas_R,
+        workspace=workspace, stream=stream)
+
     def step(i, ev=None):
-        snap = nb.nbos_snapshot_create(w.n_snapshots, w.n_hosts, lim_num, lim_den, *d_state,
-                                       replicas_R=w.replicas_R, workspace=workspace, stream=stream)
+        if live is None:
+            snap = nb.nbos_snapshot_create(w.n_snapshots, w.n_hosts, lim_num, lim_den, *d_state,
+                                           replicas_R=w.replicas_R, workspace=workspace, stream=stream)
+        else:
+            snap = live
+            nb.nbos_snapshot_update(snap, lim_num, lim_den, *d_state, stream=stream)
         k = i % n_rot
         if ev is not None:
             ev[0].record(stream)
@@ -240,8 +253,9 @@ def run_ours(args):
     for i in range(max(3, args.warmup)):
         snaps.append(step(i))
     sync_all()
-    for s in snaps:
-        nb.nbos_snapshot_destroy(s)
+    if live is None:
+        for s in snaps:
+            nb.nbos_snapshot_destroy(s)
     snaps = []
     kern_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
                    for _ in range(args.steps)]
@@ -254,8 +268,18 @@ def run_ours(args):
     sync_all()
     sampler.stop()
     status = nb.nbos_snapshot_status(snaps[-1], stream)
-    for s in snaps:
-        nb.nbos_snapshot_destroy(s)
+    # creation on its own, for the record (one host synchronisation inside)
+    t0 = time.perf_counter()
+    for _ in range(10):
+        nb.nbos_snapshot_destroy(nb.nbos_snapshot_create(
+            w.n_snapshots, w.n_hosts, lim_num, lim_den, *d_state, replicas_R=w.replicas_R, stream=stream))
+    torch.cuda.synchronize()
+    create_ms = (time.perf_counter() - t0) / 10 * 1e3
+    if live is None:
+        for s in snaps:
+            nb.nbos_snapshot_destroy(s)
+    else:
+        nb.nbos_snapshot_destroy(live)
     if status != nb.NBOS_OK:
         raise RuntimeError("device status: " + nb.nbos_strerror(status))
     ms_total = e0.elapsed_time(e1)
@@ -277,11 +301,19 @@ def run_ours(args):
         h_out = torch.empty((w.n_snapshots, w.batch, 3), dtype=torch.int32).pin_memory()
         h_found = torch.empty((w.n_snapshots, w.batch), dtype=torch.int32).pin_memory()
 
+        e2e_live = None if args.fresh_snapshot else nb.nbos_snapshot_create_host(
+            w.n_snapshots, w.n_hosts, lim_num, lim_den, *h_state, replicas_R=w.replicas_R, stream=stream)
+
         def e2e_step(i):
-            snap = nb.nbos_snapshot_create_host(w.n_snapshots, w.n_hosts, lim_num, lim_den,
-                                                *h_state, replicas_R=w.replicas_R, stream=stream)
+            if e2e_live is None:
+                snap = nb.nbos_snapshot_create_host(w.n_snapshots, w.n_hosts, lim_num, lim_den,
+                                                    *h_state, replicas_R=w.replicas_R, stream=stream)
+            else:
+                snap = e2e_live
+                nb.nbos_snapshot_update_host(snap, lim_num, lim_den, *h_state, stream=stream)
             nb.nbos_place_batch_host(snap, h_req[i % 2], h_out, h_found, stream=stream)
-            nb.nbos_snapshot_destroy(snap)
+            if e2e_live is None:
+                nb.nbos_snapshot_destroy(snap)
 
         e2e_steps = max(3, min(args.steps, 20))
         for i in range(3):
@@ -299,6 +331,8 @@ def run_ours(args):
         e2e_ms = float(t.item()) / e2e_steps
         h2d = w.decisions * 16 + 6 * 4 * w.n_snapshots * w.n_hosts + 8 * w.n_snapshots
         d2h = w.decisions * (12 + 4)
+        if e2e_live is not None:
+            nb.nbos_snapshot_destroy(e2e_live)
         e2e = {"value": decisions_all / (e2e_ms * 1e-3), "unit": "decisions/s",
                "ms_per_step": e2e_ms, "steps": e2e_steps, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "host_memory": "pinned"}
@@ -457,7 +491,7 @@ def run_ours(args):
             nb.nbos_snapshot_destroy(sn)
 
     rot_mib = n_rot * per_batch_bytes / 2**20
-    launches_per_step = 5  # scan, emit, rank, finalize (derivation) + placement kernel
+    launches_per_step = 5  # scan, emit, rank, finalize (derivation, same kernels for create and refresh) + placement
     line = {
         "metric": "placement decisions/sec", "value": value, "unit": "decisions/s",
         "pairs_per_s": value * w.n_hosts, "n_gpus": world, "steps": args.steps,
@@ -465,7 +499,10 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
         "config": {"workload": w.name, "n_snapshots": w.n_snapshots, "n_hosts": w.n_hosts,
                    "batch": w.batch, "pairs_per_step_per_gpu": w.pairs, "replicas_R": w.replicas_R,
-                   "step": "snapshot derivation + placement of one batch",
+                   "step": ("snapshot creation (derivation, one host synchronisation) + placement of one batch"
+                            if args.fresh_snapshot else
+                            "snapshot refresh (all derivation kernels, no read-back) + placement of one batch"),
+                   "snapshot_create_ms": create_ms,
                    "l2": f"inputs rotate over {n_rot} request/result batch sets, {rot_mib:.0f} MiB "
                          f"in total ({'larger' if rot_mib > 126 else 'SMALLER'} than the 126 MiB L2)",
                    "inputs_sha256": w.sha256()},
