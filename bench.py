@@ -377,7 +377,7 @@ def run_ours(args):
 
     cpu_baseline = None
     if not args.no_cpu_baseline:
-        sample = args.cpu_sample or max(16, min(w.batch, (1 << 28) // (w.n_snapshots * w.n_hosts)))
+        sample = args.cpu_sample or max(16, min(w.batch, (1 << 30) // (w.n_snapshots * w.n_hosts)))
         dec, dt, res = time_checker(w, sample, 1, 0)
         same = bool(np.array_equal(res[0], d_out[0][:, :sample].cpu().numpy())
                     and np.array_equal(res[1], d_found[0][:, :sample].cpu().numpy()))
