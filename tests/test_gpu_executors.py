@@ -50,7 +50,7 @@ def cpu_select(w, req, rep):
 @pytest.mark.parametrize("maker", [lambda: W.make_config(1), lambda: W.make_config(2),
                                    lambda: W.mixed_gpu_cluster(500, 16, seed=5),
                                    lambda: W.uniform_cluster(3, 16, seed=6)])
-@pytest.mark.parametrize("m", [1, 1000, 300_001])
+@pytest.mark.parametrize("m", [1, 1000, 300_001, 1_300_003])
 def test_executor_selection_matches_the_checker(nb, maker, m):
     w = maker()
     rng = np.random.default_rng(m)
