@@ -136,7 +136,11 @@ typedef struct nbos_snapshot_info {
  *   pair_mode          how a (request, host) pair is evaluated when the snapshot has 32-bit keys:
  *                      0 = the fastest form the snapshot allows; 1 = four separate capacity
  *                      compares; 2 = packed capacity test with the key computed per pair (even if
- *                      the snapshot would allow ranking by the host part of the key alone).
+ *                      the snapshot would allow ranking by the host part of the key alone);
+ *                      3 = packed capacity test with the host part of the key compared per pair
+ *                      (even if the table is stored in key order, where 0 drops that compare:
+ *                      a feasible host then enters a request's best three exactly while the
+ *                      request has fewer than three). Every form gives the same outputs.
  *   first_fit          1 = stop scanning a request's hosts at the third feasible one. Possible
  *                      when every host has the same key slope and the table is stored in key
  *                      order (nbos_snapshot_info: static_key and presorted), because then the

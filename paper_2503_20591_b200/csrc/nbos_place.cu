@@ -43,10 +43,16 @@ enum : int {
     MODE_PACKED_STATIC = 3,  // as 2, but B is the same on every host: rank by A alone (records: pk)
     MODE_PACKED2 = 4,        // as 2, the two words have their low guard bit at different positions
     MODE_PACKED2_STATIC = 5, // as 3, likewise
-    MODE_COUNT = 6,
+    MODE_SORTED = 6,         // as 3, and the records are stored in ascending key order: a feasible host
+                             // enters the best three exactly while the request has fewer than three,
+                             // so the key compare is replaced by retiring the request's packed words
+    MODE_SORTED2 = 7,        // as 6 with two guard masks
+    MODE_COUNT = 8,
 };
 __host__ __device__ constexpr bool mode_is_packed(int mode) { return mode >= MODE_PACKED; }
-__host__ __device__ constexpr bool mode_is_static(int mode) { return mode == MODE_PACKED_STATIC || mode == MODE_PACKED2_STATIC; }
+__host__ __device__ constexpr bool mode_is_sorted(int mode) { return mode == MODE_SORTED || mode == MODE_SORTED2; }
+__host__ __device__ constexpr bool mode_is_static(int mode) { return mode == MODE_PACKED_STATIC || mode == MODE_PACKED2_STATIC || mode_is_sorted(mode); }
+__host__ __device__ constexpr bool mode_two_masks(int mode) { return mode == MODE_PACKED2 || mode == MODE_PACKED2_STATIC || mode == MODE_SORTED2; }
 __host__ __device__ constexpr int mode_record_bytes(int mode) { return mode == MODE_KEY64 ? 32 : mode == MODE_PLAIN ? 24 : 16; }
 __host__ __device__ constexpr int mode_max_q(int mode) { return mode == MODE_KEY64 ? 4 : 8; }
 constexpr int kStages = 3;
@@ -215,6 +221,34 @@ __device__ __forceinline__ void pair_packed2_static(float &cnt, unsigned int t3,
         : "r"(t3), "r"(r0), "r"(r1), "r"(h.x), "r"(h.y), "r"(h.z), "r"(guards0), "r"(guards1));
 }
 
+// Sorted forms: the capacity test alone decides; a request that has its three hosts carries
+// packed words that fail against every host (see run_pass).
+__device__ __forceinline__ void pair_sorted(float &cnt, unsigned int r0, unsigned int r1, const uint4 &h,
+                                            unsigned int guards)
+{
+    asm volatile(
+        "{\n\t.reg .pred bad;\n\t.reg .u32 d0, d1, e;\n\t"
+        "mad.lo.u32 d0, %1, 0xffffffff, %3;\n\t"
+        "mad.lo.u32 d1, %2, 0xffffffff, %4;\n\t"
+        "lop3.and.b32 e|bad, d0, d1, %5, 0x2a, 1;\n\t"
+        "@!bad add.f32 %0, %0, 0f3F800000;\n\t}"
+        : "+f"(cnt)
+        : "r"(r0), "r"(r1), "r"(h.x), "r"(h.y), "r"(guards));
+}
+__device__ __forceinline__ void pair_sorted2(float &cnt, unsigned int r0, unsigned int r1, const uint4 &h,
+                                             unsigned int guards0, unsigned int guards1)
+{
+    asm volatile(
+        "{\n\t.reg .pred bad;\n\t.reg .u32 d0, d1, e0, e;\n\t"
+        "mad.lo.u32 d0, %1, 0xffffffff, %3;\n\t"
+        "mad.lo.u32 d1, %2, 0xffffffff, %4;\n\t"
+        "lop3.b32 e0, d0, %5, 0, 0x0c;\n\t"
+        "lop3.and.b32 e|bad, e0, d1, %6, 0xf2, 1;\n\t"
+        "@!bad add.f32 %0, %0, 0f3F800000;\n\t}"
+        : "+f"(cnt)
+        : "r"(r0), "r"(r1), "r"(h.x), "r"(h.y), "r"(guards0), "r"(guards1));
+}
+
 template <int MODE> struct ModeTraits {
     using Key = unsigned int;
     using Pair = uint2;
@@ -345,6 +379,8 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
                         if (MODE == MODE_PACKED) pair_packed(cnt, (unsigned int)t3[q], r0[q], r1[q], (unsigned int)g[q], h[u], guards0);
                         else if (MODE == MODE_PACKED_STATIC) pair_packed_static(cnt, (unsigned int)t3[q], r0[q], r1[q], h[u], guards0);
                         else if (MODE == MODE_PACKED2) pair_packed2(cnt, (unsigned int)t3[q], r0[q], r1[q], (unsigned int)g[q], h[u], guards0, guards1);
+                        else if (MODE == MODE_SORTED) pair_sorted(cnt, r0[q], r1[q], h[u], guards0);
+                        else if (MODE == MODE_SORTED2) pair_sorted2(cnt, r0[q], r1[q], h[u], guards0, guards1);
                         else pair_packed2_static(cnt, (unsigned int)t3[q], r0[q], r1[q], h[u], guards0, guards1);
                     }
                 if (cnt != seen) {
@@ -358,6 +394,13 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
                             const unsigned int key = mode_is_static(MODE) ? h[u].z : (unsigned int)g[q] * h[u].w + h[u].z;
                             insert3(t1[q], t2[q], t3[q], (KeyT)(bad ? 0xFFFFFFFFu : key));
                         }
+                    if (mode_is_sorted(MODE)) {
+                        // three hosts found: every later host has a larger key. Retire the request
+                        // with a word equal to the guard mask, which clears every guard of any host
+#pragma unroll
+                        for (int q = 0; q < Q; ++q)
+                            if (t3[q] != kInf) r0[q] = guards0;
+                    }
                 }
             };
             int i = sub;
@@ -557,6 +600,8 @@ struct FirstFitParams {
 __global__ void __launch_bounds__(256) place_first_fit_kernel(const FirstFitParams p)
 {
     constexpr int kLanes = 8;
+    constexpr int kGroupHosts = 32;  // hosts a group looks at before the warp takes over
+    constexpr int kWide = 4;         // 32-host rows the warp loads per step once it has taken over
     const int lane = threadIdx.x & 31;
     const int sub = lane & (kLanes - 1);
     const int grp_in_warp = lane / kLanes;
@@ -564,11 +609,15 @@ __global__ void __launch_bounds__(256) place_first_fit_kernel(const FirstFitPara
     const long long my_group = (long long)blockIdx.x * (blockDim.x / kLanes) + threadIdx.x / kLanes;
     // all four groups of a warp make the same number of rounds, so that the ballots stay warp-wide
     const long long rounds = (p.n_req + groups_total - 1) / groups_total;
+    // the next round's request is fetched while this round walks its hosts
+    int4 q_next = my_group < p.n_req ? __ldg(p.requests + p.first_req + my_group) : make_int4(-1, 0, 0, 0);
     for (long long round = 0; round < rounds; ++round) {
         const long long idx = round * groups_total + my_group;
         const bool live = idx < p.n_req;
         const long long r = p.first_req + (live ? idx : 0);
-        const int4 q = live ? __ldg(p.requests + r) : make_int4(-1, 0, 0, 0);
+        const int4 q = q_next;
+        if (idx + groups_total < p.n_req) q_next = __ldg(p.requests + r + groups_total);
+        else q_next = make_int4(-1, 0, 0, 0);
         const size_t row = (size_t)(r / p.B) * p.Hpad;
         bool sane = (q.x | q.y | q.z | q.w) >= 0;
         unsigned int w0 = 0u, w1 = 0u;
@@ -581,30 +630,67 @@ __global__ void __launch_bounds__(256) place_first_fit_kernel(const FirstFitPara
                 if (p.pack.fword[k]) w1 |= piece; else w0 |= piece;
             }
         }
+        // one host test, shared by both phases
+        auto fits_host = [&](const int4 &qq, unsigned int ww0, unsigned int ww1, size_t rrow, int i,
+                             unsigned int &id) -> bool {
+            if (p.pack.enabled) {
+                const uint4 h = __ldg(p.pk + rrow + i);
+                const unsigned int d0 = h.x - ww0, d1 = h.y - ww1;
+                id = h.z & p.id_mask;
+                return ((~d0 & p.pack.guards) | (~d1 & p.pack.guards1)) == 0u;
+            }
+            const int4 f = __ldg(p.feas + rrow + i);
+            id = (p.key64 ? (unsigned int)__ldg(reinterpret_cast<const ulonglong2 *>(p.ab) + rrow + i).x
+                          : __ldg(reinterpret_cast<const uint2 *>(p.ab) + rrow + i).x) & p.id_mask;
+            return qq.x <= f.x && qq.y <= f.y && qq.z <= f.z && qq.w <= f.w;
+        };
+
+        // phase 1: the group's 8 lanes test 8 hosts per step over the first kGroupHosts hosts;
+        // most requests find their three hosts there
         int found = 0;
         bool need = live && sane;
-        for (int base = 0; __ballot_sync(0xFFFFFFFFu, need) != 0u; base += kLanes) {
+        for (int base = 0; base < kGroupHosts && __ballot_sync(0xFFFFFFFFu, need) != 0u; base += kLanes) {
             const int i = base + sub;
-            bool ok = false;
             unsigned int id = 0u;
-            if (need && i < p.Hpad) {
-                if (p.pack.enabled) {
-                    const uint4 h = __ldg(p.pk + row + i);
-                    const unsigned int d0 = h.x - w0, d1 = h.y - w1;
-                    ok = ((~d0 & p.pack.guards) | (~d1 & p.pack.guards1)) == 0u;
-                    id = h.z & p.id_mask;
-                } else {
-                    const int4 f = __ldg(p.feas + row + i);
-                    ok = q.x <= f.x && q.y <= f.y && q.z <= f.z && q.w <= f.w;
-                    id = (p.key64 ? (unsigned int)__ldg(reinterpret_cast<const ulonglong2 *>(p.ab) + row + i).x
-                                  : __ldg(reinterpret_cast<const uint2 *>(p.ab) + row + i).x) & p.id_mask;
-                }
-            }
+            const bool ok = need && i < p.Hpad && fits_host(q, w0, w1, row, i, id);
             const unsigned int fits = (__ballot_sync(0xFFFFFFFFu, ok) >> (grp_in_warp * kLanes)) & ((1u << kLanes) - 1u);
             const int slot = found + __popc(fits & ((1u << sub) - 1u));
             if (ok && slot < NBOS_REPLICAS_PLACED) p.out_hosts[r * 3 + slot] = (int)id;
             found += __popc(fits);
             need = need && found < NBOS_REPLICAS_PLACED && base + kLanes < p.Hpad;
+        }
+        // phase 2: requests that are still short get the whole warp, 32 hosts per step, one
+        // request after the other (a long walk with 8 lanes would hold up the other three groups)
+#pragma unroll 1
+        for (int g = 0; g < 32 / kLanes; ++g) {
+            const int src = g * kLanes;
+            if (!__shfl_sync(0xFFFFFFFFu, (int)need, src)) continue;      // uniform across the warp
+            const int4 qq = make_int4(__shfl_sync(0xFFFFFFFFu, q.x, src), __shfl_sync(0xFFFFFFFFu, q.y, src),
+                                      __shfl_sync(0xFFFFFFFFu, q.z, src), __shfl_sync(0xFFFFFFFFu, q.w, src));
+            const unsigned int ww0 = __shfl_sync(0xFFFFFFFFu, w0, src), ww1 = __shfl_sync(0xFFFFFFFFu, w1, src);
+            const long long rr = __shfl_sync(0xFFFFFFFFu, r, src);
+            const size_t rrow = (size_t)(rr / p.B) * p.Hpad;
+            int ff = __shfl_sync(0xFFFFFFFFu, found, src);
+            // four independent loads per step: the walk is bound by load latency, and looking at
+            // up to 96 hosts too many costs nothing
+            for (int base = kGroupHosts; base < p.Hpad && ff < NBOS_REPLICAS_PLACED; base += 32 * kWide) {
+                bool ok[kWide];
+                unsigned int id[kWide];
+#pragma unroll
+                for (int u = 0; u < kWide; ++u) {
+                    const int i = base + u * 32 + lane;
+                    id[u] = 0u;
+                    ok[u] = i < p.Hpad && fits_host(qq, ww0, ww1, rrow, i, id[u]);
+                }
+#pragma unroll
+                for (int u = 0; u < kWide; ++u) {
+                    const unsigned int fits = __ballot_sync(0xFFFFFFFFu, ok[u]);
+                    const int slot = ff + __popc(fits & ((1u << lane) - 1u));
+                    if (ok[u] && slot < NBOS_REPLICAS_PLACED) p.out_hosts[rr * 3 + slot] = (int)id[u];
+                    ff += __popc(fits);
+                }
+            }
+            if (grp_in_warp == g) found = ff;
         }
         if (found > NBOS_REPLICAS_PLACED) found = NBOS_REPLICAS_PLACED;
         if (live) {
@@ -639,6 +725,8 @@ KernelFn pick_kernel(int mode, int L)
         case MODE_PACKED_STATIC: return pick_kernel_l<MODE_PACKED_STATIC>(L);
         case MODE_PACKED2: return pick_kernel_l<MODE_PACKED2>(L);
         case MODE_PACKED2_STATIC: return pick_kernel_l<MODE_PACKED2_STATIC>(L);
+        case MODE_SORTED: return pick_kernel_l<MODE_SORTED>(L);
+        case MODE_SORTED2: return pick_kernel_l<MODE_SORTED2>(L);
     }
     return nullptr;
 }
@@ -649,7 +737,8 @@ int snapshot_mode(const nbos_snapshot *s, int forced)
     if (forced == 1 || !s->pack.enabled) return MODE_PLAIN;
     const bool two = s->pack.guards != s->pack.guards1;
     if (forced == 2 || !s->key.static_key) return two ? MODE_PACKED2 : MODE_PACKED;
-    return two ? MODE_PACKED2_STATIC : MODE_PACKED_STATIC;
+    if (forced == 3 || !s->presorted) return two ? MODE_PACKED2_STATIC : MODE_PACKED_STATIC;
+    return two ? MODE_SORTED2 : MODE_SORTED;
 }
 
 void fill_params(PlaceParams &p, const nbos_snapshot *s, const int32_t *d_requests, int64_t batch,
@@ -679,7 +768,7 @@ bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
 // What launch_place decides before it looks at the host split: evaluation mode, tile size,
 // shared memory, resident blocks per SM and lanes per request.
 struct LaunchPlan {
-    int mode, T, tiles_total, per_sm, L;
+    int mode, T, tiles_total, per_sm, blocks_per_sm, L;
     size_t smem;
 };
 
@@ -703,28 +792,44 @@ int make_plan(const nbos_snapshot *s, long long total, const nbos_launch_config 
     NBOS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn1, kThreads, smem));
     if (per_sm < 1) return fail(NBOS_ERR_CUDA, "placement kernel does not fit on an SM (%zu bytes of shared memory)", smem);
 
-    // Lanes per request: estimate, for each L, the pair steps one lane of the busiest block has to
-    // make (passes in units of requests per lane, weighted by how well a pass of that size
-    // amortises the per-host overhead, times hosts per lane) plus the shuffle merges, and take
-    // the cheapest. Large batches end up with few lanes, small ones with a whole warp.
+    // Lanes per request and resident blocks per SM: estimate, for each choice, the pair steps the
+    // busiest SM has to issue (per block: passes in units of requests per lane, weighted by how
+    // well a pass of that size amortises the per-host overhead, times hosts per lane, plus the
+    // shuffle merges; times the blocks the SM holds) and take the cheapest. Large batches end up
+    // with few lanes, small ones with a whole warp. Fewer blocks than fit can win because each
+    // block then gets more requests and its last pass is fuller; a single block per SM has too
+    // few warps to keep the issue slots busy, which the penalty accounts for.
     int L = c.lanes_per_request;
-    if (!L) {
-        const long long slots = (long long)s->sm_count * per_sm;
+    int blocks_per_sm = per_sm;
+    {
         double best = 0.0;
+        bool have = false;
         for (int cand = 1, lg = 0; cand <= 32; cand <<= 1, ++lg) {
+            if (c.lanes_per_request && cand != c.lanes_per_request) continue;
             const long long groups = kComputeThreads / cand;
-            long long ctas = (total + groups - 1) / groups;
-            if (ctas > slots) ctas = slots;
-            const long long n_req = (total + ctas - 1) / ctas;
-            const long long full = n_req / (groups * max_q_kernel), rem = n_req % (groups * max_q_kernel);
-            int q = max_q_kernel;
-            while (q > 2 && (long long)(q >> 1) * groups >= rem) q >>= 1;
-            const double weight = q >= 8 ? 1.0 : q == 4 ? 1.12 : 1.4;
-            const double units = (double)full * max_q_kernel + (rem ? q * weight : 0.0);
-            const double cost = units * ((double)s->Hpad / cand) + (double)(full + (rem ? 1 : 0)) * lg * max_q_kernel * 4.0;
-            if (cand == 1 || cost < best * 0.98) {
-                best = cost;
-                L = cand;
+            for (int j = per_sm; j >= 1; --j) {
+                const long long slots = (long long)s->sm_count * j;
+                long long ctas = (total + groups - 1) / groups;
+                if (ctas > slots) ctas = slots;
+                const long long n_req = (total + ctas - 1) / ctas;
+                const long long full = n_req / (groups * max_q_kernel), rem = n_req % (groups * max_q_kernel);
+                int q = max_q_kernel;
+                while (q > 2 && (long long)(q >> 1) * groups >= rem) q >>= 1;
+                const double weight = q >= 8 ? 1.0 : q == 4 ? 1.12 : 1.4;
+                const double units = (double)full * max_q_kernel + (rem ? q * weight : 0.0);
+                const long long on_sm = (ctas + s->sm_count - 1) / s->sm_count;
+                const double thin = on_sm == 1 ? 1.3 : on_sm == 2 ? 1.02 : 1.0;
+                // measured with full passes: sharing a request among lanes costs a little beyond the
+                // merges (more, shorter passes: request loads, result stores, tile hand-overs)
+                const double shared[6] = {1.0, 1.06, 1.08, 1.135, 1.2, 1.28};
+                const double cost = (double)on_sm * thin * shared[lg] *
+                                    (units * ((double)s->Hpad / cand) + (double)(full + (rem ? 1 : 0)) * lg * max_q_kernel * 4.0);
+                if (!have || cost < best * 0.98) {
+                    have = true;
+                    best = cost;
+                    L = cand;
+                    blocks_per_sm = j;
+                }
             }
         }
     }
@@ -732,6 +837,7 @@ int make_plan(const nbos_snapshot *s, long long total, const nbos_launch_config 
     plan.T = T;
     plan.tiles_total = tiles_total;
     plan.per_sm = per_sm;
+    plan.blocks_per_sm = blocks_per_sm;
     plan.L = L;
     plan.smem = smem;
     return NBOS_OK;
@@ -771,8 +877,8 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
         return fail(NBOS_ERR_INVALID_ARG, "requests_per_lane must be 1,2,4 or 8");
     if (c.host_split < 0 || c.grid_blocks < 0 || c.tile_hosts < 0 || (c.tile_hosts & 31))
         return fail(NBOS_ERR_INVALID_ARG, "launch config: negative field or tile_hosts not a multiple of 32");
-    if (c.pair_mode < 0 || c.pair_mode > 2)
-        return fail(NBOS_ERR_INVALID_ARG, "pair_mode must be 0 (automatic), 1 (plain compares) or 2 (packed, key computed per pair)");
+    if (c.pair_mode < 0 || c.pair_mode > 3)
+        return fail(NBOS_ERR_INVALID_ARG, "pair_mode must be 0 (automatic), 1 (plain compares), 2 (packed, key computed per pair) or 3 (packed, host key compared per pair)");
 
     if (c.first_fit && s->key.static_key && s->presorted) {
         FirstFitParams fp;
@@ -827,6 +933,7 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
 
     const int groups = kComputeThreads / L;
     long long req_ctas = (total + groups - 1) / groups;  // at least one request per group
+    if (per_sm > plan.blocks_per_sm && K == 1) per_sm = plan.blocks_per_sm;
     long long cap = (long long)s->sm_count * per_sm / K;
     if (cap < 1) cap = 1;
     if (c.grid_blocks) cap = c.grid_blocks;

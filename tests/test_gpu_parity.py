@@ -129,7 +129,7 @@ def test_key_widths_orders_flags(nb, lib_flags, key_order, flags):
             assert_same(got, ref, f"{w.name} order={key_order} flags={flags} lib={lib_flags}")
 
 
-@pytest.mark.parametrize("pair_mode", [0, 1, 2])
+@pytest.mark.parametrize("pair_mode", [0, 1, 2, 3])
 @pytest.mark.parametrize("lanes", [0, 1, 4, 32])
 def test_pair_evaluation_modes(nb, pair_mode, lanes):
     """Plain compares, packed test with per-pair key, and the automatic choice give the same bytes."""
