@@ -389,7 +389,7 @@ int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_hos
     // launch are as busy as in a single launch), about six chunks
     int lanes = 0;
     long long unit = 0;
-    rc = place_chunk_unit(snap, total, &lanes, &unit);
+    rc = place_chunk_unit(snap, total, batch_per_snapshot, &lanes, &unit);
     if (rc) {
         cudaFreeAsync(buf, stream);
         return rc;

@@ -27,6 +27,7 @@
 
 #include "nbos_internal.h"
 #include "nbos_ptx.cuh"
+#include "nbos_sorted_chunk.cuh"
 
 namespace nbos {
 namespace {
@@ -55,6 +56,9 @@ __host__ __device__ constexpr bool mode_is_static(int mode) { return mode == MOD
 __host__ __device__ constexpr bool mode_two_masks(int mode) { return mode == MODE_PACKED2 || mode == MODE_PACKED2_STATIC || mode == MODE_SORTED2; }
 __host__ __device__ constexpr int mode_record_bytes(int mode) { return mode == MODE_KEY64 ? 32 : mode == MODE_PLAIN ? 24 : 16; }
 __host__ __device__ constexpr int mode_max_q(int mode) { return mode == MODE_KEY64 ? 4 : 8; }
+// Resident blocks per SM the kernels are compiled for. The key-order modes touch their best-three
+// registers only on the rare update path, so 64 registers (a few spills there) buy a fourth block.
+__host__ __device__ constexpr int mode_blocks_per_sm(int mode) { return mode_is_sorted(mode) ? 4 : mode_is_static(mode) ? 3 : 2; }
 constexpr int kStages = 3;
 
 struct PlaceParams {
@@ -73,6 +77,7 @@ struct PlaceParams {
     int tile_hosts, tiles_total, K, req_ctas;
     unsigned int id_mask;
     int max_q;
+    unsigned int zero;      // always 0; a value the compiler cannot fold (see nbos_sorted_chunk.cuh)
 };
 
 template <typename KeyT> struct KeyTraits;
@@ -221,34 +226,6 @@ __device__ __forceinline__ void pair_packed2_static(float &cnt, unsigned int t3,
         : "r"(t3), "r"(r0), "r"(r1), "r"(h.x), "r"(h.y), "r"(h.z), "r"(guards0), "r"(guards1));
 }
 
-// Sorted forms: the capacity test alone decides; a request that has its three hosts carries
-// packed words that fail against every host (see run_pass).
-__device__ __forceinline__ void pair_sorted(float &cnt, unsigned int r0, unsigned int r1, const uint4 &h,
-                                            unsigned int guards)
-{
-    asm volatile(
-        "{\n\t.reg .pred bad;\n\t.reg .u32 d0, d1, e;\n\t"
-        "mad.lo.u32 d0, %1, 0xffffffff, %3;\n\t"
-        "mad.lo.u32 d1, %2, 0xffffffff, %4;\n\t"
-        "lop3.and.b32 e|bad, d0, d1, %5, 0x2a, 1;\n\t"
-        "@!bad add.f32 %0, %0, 0f3F800000;\n\t}"
-        : "+f"(cnt)
-        : "r"(r0), "r"(r1), "r"(h.x), "r"(h.y), "r"(guards));
-}
-__device__ __forceinline__ void pair_sorted2(float &cnt, unsigned int r0, unsigned int r1, const uint4 &h,
-                                             unsigned int guards0, unsigned int guards1)
-{
-    asm volatile(
-        "{\n\t.reg .pred bad;\n\t.reg .u32 d0, d1, e0, e;\n\t"
-        "mad.lo.u32 d0, %1, 0xffffffff, %3;\n\t"
-        "mad.lo.u32 d1, %2, 0xffffffff, %4;\n\t"
-        "lop3.b32 e0, d0, %5, 0, 0x0c;\n\t"
-        "lop3.and.b32 e|bad, e0, d1, %6, 0xf2, 1;\n\t"
-        "@!bad add.f32 %0, %0, 0f3F800000;\n\t}"
-        : "+f"(cnt)
-        : "r"(r0), "r"(r1), "r"(h.x), "r"(h.y), "r"(guards0), "r"(guards1));
-}
-
 template <int MODE> struct ModeTraits {
     using Key = unsigned int;
     using Pair = uint2;
@@ -366,27 +343,33 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
         } else {
             const uint4 *R = reinterpret_cast<const uint4 *>(stage);
             const unsigned int guards0 = p.pack.guards, guards1 = p.pack.guards1;
+            const unsigned int opaque_zero = p.zero;
             float cnt = 0.f, seen = 0.f;
             auto chunk = [&](auto width, int i0) {
                 constexpr int W = decltype(width)::value;
                 uint4 h[W];
 #pragma unroll
                 for (int u = 0; u < W; ++u) h[u] = R[i0 + u * L];
-#pragma unroll
-                for (int u = 0; u < W; ++u)
-#pragma unroll
-                    for (int q = 0; q < Q; ++q) {
-                        if (MODE == MODE_PACKED) pair_packed(cnt, (unsigned int)t3[q], r0[q], r1[q], (unsigned int)g[q], h[u], guards0);
-                        else if (MODE == MODE_PACKED_STATIC) pair_packed_static(cnt, (unsigned int)t3[q], r0[q], r1[q], h[u], guards0);
-                        else if (MODE == MODE_PACKED2) pair_packed2(cnt, (unsigned int)t3[q], r0[q], r1[q], (unsigned int)g[q], h[u], guards0, guards1);
-                        else if (MODE == MODE_SORTED) pair_sorted(cnt, r0[q], r1[q], h[u], guards0);
-                        else if (MODE == MODE_SORTED2) pair_sorted2(cnt, r0[q], r1[q], h[u], guards0, guards1);
-                        else pair_packed2_static(cnt, (unsigned int)t3[q], r0[q], r1[q], h[u], guards0, guards1);
-                    }
-                if (cnt != seen) {
-                    seen = cnt;
+                bool hit;  // some pair of the chunk may enter its request's best three
+                if constexpr (mode_is_sorted(MODE)) {
+                    // table in key order: the capacity test alone decides (chained predicate)
+                    hit = sorted_chunk_any_fit<Q, W, mode_two_masks(MODE)>(r0, r1, h, guards0, guards1, opaque_zero);
+                } else {
 #pragma unroll
                     for (int u = 0; u < W; ++u)
+#pragma unroll
+                        for (int q = 0; q < Q; ++q) {
+                            if (MODE == MODE_PACKED) pair_packed(cnt, (unsigned int)t3[q], r0[q], r1[q], (unsigned int)g[q], h[u], guards0);
+                            else if (MODE == MODE_PACKED_STATIC) pair_packed_static(cnt, (unsigned int)t3[q], r0[q], r1[q], h[u], guards0);
+                            else if (MODE == MODE_PACKED2) pair_packed2(cnt, (unsigned int)t3[q], r0[q], r1[q], (unsigned int)g[q], h[u], guards0, guards1);
+                            else pair_packed2_static(cnt, (unsigned int)t3[q], r0[q], r1[q], h[u], guards0, guards1);
+                        }
+                    hit = cnt != seen;
+                    seen = cnt;
+                }
+                if (hit) {
+#pragma unroll
+                    for (int u = 0; u < W; ++u) {
 #pragma unroll
                         for (int q = 0; q < Q; ++q) {
                             const unsigned int d0 = h[u].x - r0[q], d1 = h[u].y - r1[q];
@@ -394,6 +377,7 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
                             const unsigned int key = mode_is_static(MODE) ? h[u].z : (unsigned int)g[q] * h[u].w + h[u].z;
                             insert3(t1[q], t2[q], t3[q], (KeyT)(bad ? 0xFFFFFFFFu : key));
                         }
+                    }
                     if (mode_is_sorted(MODE)) {
                         // three hosts found: every later host has a larger key. Retire the request
                         // with a word equal to the guard mask, which clears every guard of any host
@@ -448,7 +432,7 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
 }
 
 template <int L, int MODE>
-__global__ void __launch_bounds__(kThreads, mode_is_static(MODE) ? 3 : 2)
+__global__ void __launch_bounds__(kThreads, mode_blocks_per_sm(MODE))
 place_kernel(const __grid_constant__ PlaceParams p)
 {
     constexpr int MAXQ = mode_max_q(MODE);
@@ -760,6 +744,7 @@ void fill_params(PlaceParams &p, const nbos_snapshot *s, const int32_t *d_reques
     p.N = s->N;
     p.Hpad = s->Hpad;
     p.id_mask = (1u << s->key.bits_id) - 1u;
+    p.zero = 0u;
 }
 
 bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
@@ -772,7 +757,8 @@ struct LaunchPlan {
     size_t smem;
 };
 
-int make_plan(const nbos_snapshot *s, long long total, const nbos_launch_config &c, LaunchPlan &plan)
+int make_plan(const nbos_snapshot *s, long long total, long long batch, const nbos_launch_config &c,
+              LaunchPlan &plan)
 {
     const int mode = snapshot_mode(s, c.pair_mode);
     const int record = mode_record_bytes(mode);
@@ -792,39 +778,53 @@ int make_plan(const nbos_snapshot *s, long long total, const nbos_launch_config 
     NBOS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn1, kThreads, smem));
     if (per_sm < 1) return fail(NBOS_ERR_CUDA, "placement kernel does not fit on an SM (%zu bytes of shared memory)", smem);
 
-    // Lanes per request and resident blocks per SM: estimate, for each choice, the pair steps the
-    // busiest SM has to issue (per block: passes in units of requests per lane, weighted by how
-    // well a pass of that size amortises the per-host overhead, times hosts per lane, plus the
-    // shuffle merges; times the blocks the SM holds) and take the cheapest. Large batches end up
-    // with few lanes, small ones with a whole warp. Fewer blocks than fit can win because each
-    // block then gets more requests and its last pass is fuller; a single block per SM has too
-    // few warps to keep the issue slots busy, which the penalty accounts for.
+    // Lanes per request and resident blocks per SM: for each choice, estimate the instructions a
+    // compute warp of the busiest SM issues -- per pass a fixed part, a part per request of a lane
+    // (load, packing, best-three updates, result store), a part per host of a lane and the pair
+    // steps proper, plus the shuffle merges -- and divide by the issue rate the SM reaches with
+    // that many resident blocks. The constants were fitted to timings of the five benchmark
+    // shapes and of shrunk batches over all (lanes, blocks per SM) choices. Large batches end up
+    // with one lane per request, small ones with a whole warp; fewer blocks than fit can win
+    // because each block then gets more requests and its last pass is fuller.
     int L = c.lanes_per_request;
     int blocks_per_sm = per_sm;
     {
+        const double pair_cost = mode_is_sorted(mode) ? 3.0 : mode_is_static(mode) ? 4.0 : mode_is_packed(mode) ? 5.0
+                                 : mode == MODE_PLAIN ? 7.0 : 12.0;
+        const double kPassCost = 490.0, kRequestCost = 190.0, kHostCost = 1.6, kMergeCost = 12.0;
+        const double issue_rate[4] = {0.376, 0.472, 0.499, 0.529};  // per scheduler, by resident blocks
+        const long long B = batch > 0 ? batch : total;
         double best = 0.0;
         bool have = false;
         for (int cand = 1, lg = 0; cand <= 32; cand <<= 1, ++lg) {
             if (c.lanes_per_request && cand != c.lanes_per_request) continue;
             const long long groups = kComputeThreads / cand;
+            const double per_host = (double)s->Hpad / cand;
             for (int j = per_sm; j >= 1; --j) {
                 const long long slots = (long long)s->sm_count * j;
                 long long ctas = (total + groups - 1) / groups;
                 if (ctas > slots) ctas = slots;
-                const long long n_req = (total + ctas - 1) / ctas;
-                const long long full = n_req / (groups * max_q_kernel), rem = n_req % (groups * max_q_kernel);
-                int q = max_q_kernel;
-                while (q > 2 && (long long)(q >> 1) * groups >= rem) q >>= 1;
-                const double weight = q >= 8 ? 1.0 : q == 4 ? 1.12 : 1.4;
-                const double units = (double)full * max_q_kernel + (rem ? q * weight : 0.0);
+                long long n_req = (total + ctas - 1) / ctas;
+                n_req = (n_req + 31) / 32 * 32;
+                // the block's range is cut at snapshot boundaries, each piece into passes
+                double instr = 0.0;
+                const long long pieces = n_req > B ? n_req / B : 1;
+                const long long piece_len = n_req > B ? B : n_req, tail_len = n_req > B ? n_req % B : 0;
+                for (int part = 0; part < 2; ++part) {
+                    const long long len = part ? tail_len : piece_len, times = part ? 1 : pieces;
+                    if (len <= 0) continue;
+                    const long long full = len / (groups * max_q_kernel), rem = len % (groups * max_q_kernel);
+                    int q = max_q_kernel;
+                    while (q > 2 && (long long)(q >> 1) * groups >= rem) q >>= 1;
+                    auto pass = [&](int qq) {
+                        return kPassCost + qq * kRequestCost + per_host * (kHostCost + pair_cost * qq) + lg * qq * kMergeCost;
+                    };
+                    instr += (double)times * ((double)full * pass(max_q_kernel) + (rem ? pass(q) : 0.0));
+                }
                 const long long on_sm = (ctas + s->sm_count - 1) / s->sm_count;
-                const double thin = on_sm == 1 ? 1.3 : on_sm == 2 ? 1.02 : 1.0;
-                // measured with full passes: sharing a request among lanes costs a little beyond the
-                // merges (more, shorter passes: request loads, result stores, tile hand-overs)
-                const double shared[6] = {1.0, 1.06, 1.08, 1.135, 1.2, 1.28};
-                const double cost = (double)on_sm * thin * shared[lg] *
-                                    (units * ((double)s->Hpad / cand) + (double)(full + (rem ? 1 : 0)) * lg * max_q_kernel * 4.0);
-                if (!have || cost < best * 0.98) {
+                const int resident = (int)(on_sm < j ? on_sm : j);
+                const double cost = (double)on_sm * instr / issue_rate[resident > 4 ? 3 : resident - 1];
+                if (!have || cost < best * 0.99) {
                     have = true;
                     best = cost;
                     L = cand;
@@ -848,11 +848,11 @@ int make_plan(const nbos_snapshot *s, long long total, const nbos_launch_config 
 // For callers that cut a batch into several launches (the host-buffer pipeline): the lanes per
 // request the whole batch would get, and the number of requests that gives every resident block
 // exactly one full pass -- chunks that are multiples of it keep every lane busy.
-int place_chunk_unit(const nbos_snapshot *s, long long total, int *lanes, long long *unit)
+int place_chunk_unit(const nbos_snapshot *s, long long total, long long batch, int *lanes, long long *unit)
 {
     nbos_launch_config c = {};
     LaunchPlan plan;
-    int rc = make_plan(s, total, c, plan);
+    int rc = make_plan(s, total, batch, c, plan);
     if (rc) return rc;
     *lanes = plan.L;
     *unit = (long long)s->sm_count * plan.per_sm * (kComputeThreads / plan.L) * mode_max_q(plan.mode);
@@ -903,24 +903,27 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
     }
 
     LaunchPlan plan;
-    int rc = make_plan(s, total, c, plan);
+    int rc = make_plan(s, total, batch, c, plan);
     if (rc) return rc;
-    const int mode = plan.mode, T = plan.T, tiles_total = plan.tiles_total, L = plan.L;
+    const int mode = plan.mode, T = plan.T, tiles_total = plan.tiles_total;
     const int max_q_kernel = mode_max_q(mode);
     const bool k64 = mode == MODE_KEY64;
     const size_t smem = plan.smem;
     int per_sm = plan.per_sm;
-    const long long want_threads = (long long)s->sm_count * per_sm * kComputeThreads;
+    // Hosts are cut into slices only when the batch is so small that even a warp per request
+    // leaves SMs without a block.
+    const long long one_block_per_sm = (long long)s->sm_count * kComputeThreads;
     int K = c.host_split;
     if (!K) {
         K = 1;
-        if (total * L < want_threads) {
-            long long k = (want_threads + total * L - 1) / (total * L);
+        if (total * 32 < one_block_per_sm && !c.lanes_per_request) {
+            const long long k = (one_block_per_sm + total * 32 - 1) / (total * 32);
             K = (int)(k < tiles_total ? k : tiles_total);
         }
     }
     if (K > tiles_total) K = tiles_total;
     if (K < 1) K = 1;
+    const int L = (K > 1 && !c.lanes_per_request) ? 32 : plan.L;
 
     int max_q = c.requests_per_lane ? c.requests_per_lane : max_q_kernel;
     if (max_q > max_q_kernel) max_q = max_q_kernel;
