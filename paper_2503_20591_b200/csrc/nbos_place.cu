@@ -77,7 +77,6 @@ struct PlaceParams {
     int tile_hosts, tiles_total, K, req_ctas;
     unsigned int id_mask;
     int max_q;
-    unsigned int zero;      // always 0; a value the compiler cannot fold (see nbos_sorted_chunk.cuh)
 };
 
 template <typename KeyT> struct KeyTraits;
@@ -343,7 +342,6 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
         } else {
             const uint4 *R = reinterpret_cast<const uint4 *>(stage);
             const unsigned int guards0 = p.pack.guards, guards1 = p.pack.guards1;
-            const unsigned int opaque_zero = p.zero;
             float cnt = 0.f, seen = 0.f;
             auto chunk = [&](auto width, int i0) {
                 constexpr int W = decltype(width)::value;
@@ -353,7 +351,7 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
                 bool hit;  // some pair of the chunk may enter its request's best three
                 if constexpr (mode_is_sorted(MODE)) {
                     // table in key order: the capacity test alone decides (chained predicate)
-                    hit = sorted_chunk_any_fit<Q, W, mode_two_masks(MODE)>(r0, r1, h, guards0, guards1, opaque_zero);
+                    hit = sorted_chunk_any_fit<Q, W, mode_two_masks(MODE)>(r0, r1, h, guards0, guards1);
                 } else {
 #pragma unroll
                     for (int u = 0; u < W; ++u)
@@ -744,7 +742,6 @@ void fill_params(PlaceParams &p, const nbos_snapshot *s, const int32_t *d_reques
     p.N = s->N;
     p.Hpad = s->Hpad;
     p.id_mask = (1u << s->key.bits_id) - 1u;
-    p.zero = 0u;
 }
 
 bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
