@@ -35,7 +35,10 @@ ALGORITHMIC_OPS_PER_PAIR = 6      # 4 capacity compares + 1 multiply-add (key) +
 L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (read + write) of one placement-kernel launch on the default workload, from the ncu
 # capture summarised under profiles/. None while no capture matches the current kernel.
-PLACE_KERNEL_DRAM_BYTES_PER_LAUNCH = 16_914_176
+PLACE_KERNEL_DRAM_BYTES_PER_LAUNCH = 16_957_696
+# Warp instructions the placement kernel executes per 32 pairs on the default workload, from the
+# same capture (smsp__inst_executed.sum / (pairs / 32)).
+PLACE_KERNEL_WARP_INSTR_PER_32_PAIRS = 3.59
 
 
 def parse_args():
@@ -296,7 +299,7 @@ def run_ours(args):
     # ---- end to end: host buffers in, host buffers out, through the *_host entry points ----
     e2e = None
     if not args.no_e2e:
-        h_state = [torch.from_numpy(getattr(w, k)).reshape(-1) for k in w.HOST_FIELDS]
+        h_state = [torch.from_numpy(getattr(w, k)).reshape(-1).pin_memory() for k in w.HOST_FIELDS]
         h_req = [torch.from_numpy(b).pin_memory() for b in batches[:2]]
         h_out = torch.empty((w.n_snapshots, w.batch, 3), dtype=torch.int32).pin_memory()
         h_found = torch.empty((w.n_snapshots, w.batch), dtype=torch.int32).pin_memory()
@@ -363,9 +366,14 @@ def run_ours(args):
                        f"({ALU_LANES_PER_SM} ALU + {IMAD_LANES_PER_SM} multiply-pipe lanes) x "
                        f"{sm_mhz:.0f} MHz sampled during the timed region; probe_both_gops is this "
                        "peak measured in the same process, probe_alu_gops / probe_imad_gops each pipe alone",
-        "note": "achieved counts the 6 algorithmic operations of a pair; the kernel executes fewer "
-                "instructions than that (two capacity compares per packed subtraction, no multiply-add "
-                "when all hosts share the key slope), so frac_of_alu_pipe_alone can exceed 1",
+        "note": "achieved counts the 6 algorithmic operations of a pair (4 capacity compares, key multiply-add, "
+                "compare with the third best). The kernel executes about 3 instructions per pair instead: the four "
+                "compares are two packed subtractions and one logic operation, and with the host table in key "
+                "order the key never has to be computed or compared. So frac can exceed 1 without any pair being "
+                "skipped; issue_slot_frac is the executed-instruction view of the same launch",
+        "issue_slot_frac": (PLACE_KERNEL_WARP_INSTR_PER_32_PAIRS * w.pairs / 32 / (kern_ms * 1e-3)
+                            / (sms * 4 * sm_mhz * 1e6)) if (args.workload == 3 and args.batch is None) else None,
+        "warp_instructions_per_32_pairs": PLACE_KERNEL_WARP_INSTR_PER_32_PAIRS if (args.workload == 3 and args.batch is None) else None,
         "ops_per_pair": ALGORITHMIC_OPS_PER_PAIR, "kernel_ms": kern_ms,
         "pairs_per_s_kernel": w.pairs / (kern_ms * 1e-3),
         "traffic": PLACE_KERNEL_DRAM_BYTES_PER_LAUNCH if (args.workload == 3 and args.batch is None) else None,

@@ -384,21 +384,14 @@ int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_hos
     int32_t *d_found = out_found_host ? reinterpret_cast<int32_t *>(buf + up(req_bytes) + up(out_bytes)) : nullptr;
 
     // chunks of the flattened request list: copy in, place, copy out, round-robin over the side
-    // streams so that the copies of one chunk overlap the kernel of another
-    // chunk = a whole number of full passes of all resident blocks (so that the lanes of every chunk
-    // launch are as busy as in a single launch), about six chunks
-    int lanes = 0;
-    long long unit = 0;
-    rc = place_chunk_unit(snap, total, batch_per_snapshot, &lanes, &unit);
-    if (rc) {
-        cudaFreeAsync(buf, stream);
-        return rc;
-    }
-    long long passes = total / unit;            // full passes in the batch
-    long long per_chunk = passes >= 12 ? passes / 6 : passes >= 4 ? 1 : 0;
-    const long long chunk = per_chunk ? per_chunk * unit : ((total + 31) & ~31ll);
-    nbos_launch_config chunk_cfg = {};
-    chunk_cfg.lanes_per_request = lanes;
+    // streams so that the copies of one chunk overlap the kernel of another. A chunk carries at
+    // least 2^28 (request, host) pairs (some 40 us of placement), so that the kernel keeps the
+    // efficiency of a large launch; at most eight chunks. Every chunk launch plans itself.
+    const long long pairs = total * (long long)snap->Hpad;
+    long long n_chunks = pairs >> 28;
+    if (n_chunks < 1) n_chunks = 1;
+    if (n_chunks > 8) n_chunks = 8;
+    const long long chunk = (((total + n_chunks - 1) / n_chunks) + 31) & ~31ll;
     e = cudaEventRecord(pipe->start, stream);
     for (int j = 0; j < HostPipe::kStreams && e == cudaSuccess; ++j) e = cudaStreamWaitEvent(pipe->streams[j], pipe->start, 0);
     int used = 0;
@@ -408,7 +401,7 @@ int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_hos
         if (i < HostPipe::kStreams) used = (int)i + 1;
         e = cudaMemcpyAsync(d_req + lo * 4, requests_host + lo * 4, (size_t)n * 16, cudaMemcpyHostToDevice, st);
         if (e != cudaSuccess) break;
-        rc = launch_place(snap, d_req, batch_per_snapshot, d_out, d_found, st, &chunk_cfg, lo, n);
+        rc = launch_place(snap, d_req, batch_per_snapshot, d_out, d_found, st, nullptr, lo, n);
         if (rc) break;
         e = cudaMemcpyAsync(out_hosts_host + lo * 3, d_out + lo * 3, (size_t)n * 12, cudaMemcpyDeviceToHost, st);
         if (e == cudaSuccess && d_found)

@@ -114,10 +114,6 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
                  int32_t *d_out_hosts, int32_t *d_out_found, cudaStream_t stream,
                  const nbos_launch_config *cfg, long long range_first = 0, long long range_count = -1);
 
-// Lanes per request the whole batch would get, and the request count of one full pass of all
-// resident blocks (nbos_place.cu).
-int place_chunk_unit(const nbos_snapshot *s, long long total, long long batch, int *lanes, long long *unit);
-
 // Host-split placement whose candidate buffer is a fixed array inside the module (no allocation).
 int launch_place_static(const nbos_snapshot *s, const int32_t *d_requests, int64_t batch,
                         int32_t *d_out_hosts, int32_t *d_out_found, cudaStream_t stream,

@@ -842,20 +842,6 @@ int make_plan(const nbos_snapshot *s, long long total, long long batch, const nb
 
 }  // namespace
 
-// For callers that cut a batch into several launches (the host-buffer pipeline): the lanes per
-// request the whole batch would get, and the number of requests that gives every resident block
-// exactly one full pass -- chunks that are multiples of it keep every lane busy.
-int place_chunk_unit(const nbos_snapshot *s, long long total, long long batch, int *lanes, long long *unit)
-{
-    nbos_launch_config c = {};
-    LaunchPlan plan;
-    int rc = make_plan(s, total, batch, c, plan);
-    if (rc) return rc;
-    *lanes = plan.L;
-    *unit = (long long)s->sm_count * plan.per_sm * (kComputeThreads / plan.L) * mode_max_q(plan.mode);
-    return NBOS_OK;
-}
-
 int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batch,
                  int32_t *d_out_hosts, int32_t *d_out_found, cudaStream_t stream,
                  const nbos_launch_config *cfg, long long range_first, long long range_count)

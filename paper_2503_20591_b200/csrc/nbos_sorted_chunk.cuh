@@ -10,11 +10,12 @@
 // subtraction.
 //
 // Pipe balance. 32-bit integer multiply-add (mad.lo with -1: a subtraction) runs on the
-// multiply pipe, logic operations and 64-bit subtraction on the integer ALU; both pipes take a
-// warp instruction every second cycle. Five of eight requests use two multiply-pipe
-// subtractions + one logic operation, three use one 64-bit subtraction + one logic operation:
-// 22 ALU cycles and 20 multiply-pipe cycles per 8 pairs, 21 issue slots. (All requests in the
-// first form measured 4 % slower, all in the second 15 % slower.)
+// multiply pipe, logic operations on the integer ALU; both pipes take a warp instruction every
+// second cycle, so a kernel that loads only one of them leaves half of the integer issue rate
+// unused. Five of eight requests use two multiply-pipe subtractions + one logic operation,
+// three use one 64-bit subtraction (one integer-ALU instruction when measured alone) + one
+// logic operation. The split was chosen by timing: all requests in the first form measured 4 %
+// slower, all in the second 15 % slower, half and half 3 % slower.
 //
 // One asm statement covers a whole chunk (W hosts x Q requests) because a predicate cannot
 // leave an asm statement. Operand layout (fixed, unused ones are passed as zero):
