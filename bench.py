@@ -400,8 +400,10 @@ def run_ours(args):
     others = None
     if args.all_workloads:
         others = {}
-        for idx in range(5):
-            ww = W.make_config(idx)
+        shapes = [W.make_config(idx) for idx in range(5)]
+        # not one of the five: servers with 1..8 GPUs, so that the ranking depends on the ask
+        shapes.append(W.mixed_gpu_cluster(4096, 1 << 20, seed=5, name="mixed_gpu_counts_4096x1M"))
+        for ww in shapes:
             sn = nb.snapshot_from_workload(ww, device=dev)
             rq = torch.from_numpy(ww.requests).to(dev)
             oh = torch.empty((ww.n_snapshots, ww.batch, 3), dtype=torch.int32, device=dev)
@@ -438,6 +440,7 @@ def run_ours(args):
                                "first_fit_same_output": bool(torch.equal(oh, oh2)),
                                "found_histogram": torch.bincount(of.flatten(), minlength=4).tolist(),
                                "packed_test": info.packed_test, "static_key": info.static_key,
+                               "grouped": info.grouped,
                                "note": "same inputs every launch (L2-resident), back-to-back launches"}
             nb.nbos_snapshot_destroy(sn)
 

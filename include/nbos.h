@@ -119,7 +119,8 @@ typedef struct nbos_snapshot_info {
                           * mask; 2: packed, one guard mask per word                        */
     int32_t static_key;  /* 1: every host has the same key slope, hosts rank the same for all g */
     int32_t presorted;   /* 1: the host table is stored in ascending key order              */
-    int32_t reserved;
+    int32_t grouped;     /* 1: hosts differ in GPU count; the table is stored count by count,
+                          * each group in ascending key order                               */
     int64_t workspace_bytes;
 } nbos_snapshot_info;
 

@@ -68,7 +68,7 @@ class nbos_snapshot_info(ctypes.Structure):
         ("bits_idle", ctypes.c_int32), ("bits_sr", ctypes.c_int32), ("bits_id", ctypes.c_int32),
         ("key_order", ctypes.c_int32), ("flags", ctypes.c_int32), ("replicas_R", ctypes.c_int32),
         ("packed_test", ctypes.c_int32), ("static_key", ctypes.c_int32),
-        ("presorted", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("presorted", ctypes.c_int32), ("grouped", ctypes.c_int32),
         ("workspace_bytes", ctypes.c_int64),
     ]
 

@@ -325,7 +325,7 @@ int nbos_snapshot_get_info(const nbos_snapshot *s, nbos_snapshot_info *out)
     out->packed_test = !s->pack.enabled ? 0 : s->pack.guards == s->pack.guards1 ? 1 : 2;
     out->static_key = s->key.static_key;
     out->presorted = s->presorted;
-    out->reserved = 0;
+    out->grouped = s->key.grouped;
     out->workspace_bytes = (int64_t)s->workspace_bytes;
     return NBOS_OK;
 }

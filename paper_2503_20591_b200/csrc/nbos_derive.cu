@@ -214,8 +214,10 @@ struct EmitArgs {
     int H, Hpad, R, flags, key_order;
     int idle_max;             // over all snapshots: the idle field stores idle_max - (G - C)
     int bits_idle, bits_sr, bits_id;
+    int group_major;          // 1: visiting order is (GPU count, key at g = 0) instead of the key alone
 };
 
+constexpr int kMaxGpuCountGroups = 8;  // distinct GPU counts per snapshot up to which the table is grouped
 constexpr int kSortMaxHosts = 65536;  // larger tables keep host order (ranking is quadratic in the host count)
 constexpr unsigned long long kSortNever = 0xFFFFFFFF00000000ull;  // hosts that take nothing go last (| host index)
 
@@ -254,7 +256,9 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
                 A = (idle_inv << (a.bits_sr + a.bits_id)) + (sr0 << a.bits_id) + (KeyT)h;
                 B = w << a.bits_id;
             }
-            sk = sizeof(KeyT) == 4 ? ((unsigned long long)A << 32) | (unsigned int)h : (unsigned long long)A;
+            // A carries the host index in its low bits, so both forms are unique
+            if (a.group_major) sk = ((unsigned long long)(unsigned int)G << 32) | (unsigned long long)(unsigned int)A;
+            else sk = sizeof(KeyT) == 4 ? ((unsigned long long)A << 32) | (unsigned int)h : (unsigned long long)A;
         }
     }
     a.sortkey[(size_t)n * a.Hpad + h] = sk;
@@ -442,7 +446,8 @@ int emit_tables(DeriveCtx &c)
     int4 *tmp_seq = reinterpret_cast<int4 *>(c.ws + c.lay.off_tmp_seq);
     EmitArgs ea{c.G, c.S, c.C, c.AV, c.AC, c.AM, c.limits_arg, c.limit0, k.static_key ? nullptr : d_lambda,
                 s->presorted ? perm : nullptr, tmp_feas, tmp_seq, tmp_ab, sortkey,
-                H, Hpad, s->R, s->flags, s->key_order, s->idle_max, k.bits_idle, k.bits_sr, k.bits_id};
+                H, Hpad, s->R, s->flags, s->key_order, s->idle_max, k.bits_idle, k.bits_sr, k.bits_id,
+                k.grouped};
     dim3 grid((Hpad + 255) / 256, N);
     if (k.key_bits == 32)
         emit_kernel<unsigned int, uint2><<<grid, 256, 0, c.stream>>>(ea);
@@ -539,7 +544,7 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
             if (m > sr_max) sr_max = m;
         }
     }
-    KeyLayout k;
+    KeyLayout k = {};
     k.bits_idle = bits_for((unsigned long long)idle_max);
     k.bits_sr = bits_for(sr_max);
     k.bits_id = bits_for((unsigned long long)(Hpad - 1));
@@ -548,11 +553,13 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     k.key_bits = (total_bits <= 31 && !(s->flags & NBOS_FORCE_KEY64)) ? 32 : 64;
     k.static_key = 1;
     int fmax[4] = {0, 0, 0, 0};
+    int max_distinct_g = 0;
     for (int n = 0; n < N; ++n) {
         const SnapStats &st = h_stats[n];
         int distinct_g = 0;
         for (int w = 0; w < 16; ++w) distinct_g += __builtin_popcountll(st.g_mask[w]);
         if (distinct_g > 1) k.static_key = 0;
+        if (distinct_g > max_distinct_g) max_distinct_g = distinct_g;
         if (st.max_gcap1 - 1 > fmax[0]) fmax[0] = st.max_gcap1 - 1;
         if (st.max_av > fmax[1]) fmax[1] = st.max_av;
         if (st.max_ac > fmax[2]) fmax[2] = st.max_ac;
@@ -594,6 +601,12 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     }
     s->pack = pk;
     s->presorted = Hpad <= kSortMaxHosts;
+    // Hosts with different GPU counts rank differently for different asks, but within one GPU
+    // count the order is the same for every ask. With few distinct counts the table is stored
+    // count by count, each group in key order, and the placement kernel treats every group like
+    // a table in key order.
+    s->key.grouped = (!k.static_key && k.key_bits == 32 && pk.enabled && s->presorted &&
+                      max_distinct_g <= kMaxGpuCountGroups) ? 1 : 0;
 
     // what a later nbos_snapshot_update checks the new state against
     if (!k.static_key)

@@ -52,6 +52,8 @@ struct KeyLayout {
     int key_bits;  // 32 or 64
     int bits_idle, bits_sr, bits_id;
     int static_key;  // 1 if B is the same for every host that can take a request: order = order of A
+    int grouped;     // 1 if B differs between hosts and the table is stored GPU count by GPU count,
+                     // each group in ascending order of A (set only with a packed test and 32-bit keys)
 };
 
 // Two-compares-per-subtraction encoding of the four capacity tests. Components: 0 = GPUs

@@ -48,17 +48,25 @@ enum : int {
                              // enters the best three exactly while the request has fewer than three,
                              // so the key compare is replaced by retiring the request's packed words
     MODE_SORTED2 = 7,        // as 6 with two guard masks
-    MODE_COUNT = 8,
+    MODE_GROUPED = 8,        // hosts differ in key slope (GPU count) but the table is stored count by count,
+                             // each group in ascending key order: every group is treated like a table in
+                             // key order (a request is retired for the rest of a group once it has three
+                             // hosts of that group), keys are computed only for the hosts that fit
+    MODE_GROUPED2 = 9,       // as 8 with two guard masks
+    MODE_COUNT = 10,
 };
 __host__ __device__ constexpr bool mode_is_packed(int mode) { return mode >= MODE_PACKED; }
 __host__ __device__ constexpr bool mode_is_sorted(int mode) { return mode == MODE_SORTED || mode == MODE_SORTED2; }
+__host__ __device__ constexpr bool mode_is_grouped(int mode) { return mode == MODE_GROUPED || mode == MODE_GROUPED2; }
+// modes whose pair step is the capacity test alone (chained predicate, no key work per pair)
+__host__ __device__ constexpr bool mode_is_chained(int mode) { return mode_is_sorted(mode) || mode_is_grouped(mode); }
 __host__ __device__ constexpr bool mode_is_static(int mode) { return mode == MODE_PACKED_STATIC || mode == MODE_PACKED2_STATIC || mode_is_sorted(mode); }
-__host__ __device__ constexpr bool mode_two_masks(int mode) { return mode == MODE_PACKED2 || mode == MODE_PACKED2_STATIC || mode == MODE_SORTED2; }
+__host__ __device__ constexpr bool mode_two_masks(int mode) { return mode == MODE_PACKED2 || mode == MODE_PACKED2_STATIC || mode == MODE_SORTED2 || mode == MODE_GROUPED2; }
 __host__ __device__ constexpr int mode_record_bytes(int mode) { return mode == MODE_KEY64 ? 32 : mode == MODE_PLAIN ? 24 : 16; }
 __host__ __device__ constexpr int mode_max_q(int mode) { return mode == MODE_KEY64 ? 4 : 8; }
 // Resident blocks per SM the kernels are compiled for. The key-order modes touch their best-three
 // registers only on the rare update path, so 64 registers (a few spills there) buy a fourth block.
-__host__ __device__ constexpr int mode_blocks_per_sm(int mode) { return mode_is_sorted(mode) ? 4 : mode_is_static(mode) ? 3 : 2; }
+__host__ __device__ constexpr int mode_blocks_per_sm(int mode) { return mode_is_sorted(mode) ? 4 : (mode_is_static(mode) || mode_is_grouped(mode)) ? 3 : 2; }
 constexpr int kStages = 3;
 
 struct PlaceParams {
@@ -255,6 +263,11 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
     // request registers: plain modes keep the four asks, packed modes the two packed words
     int g[Q], v[kPacked ? 1 : Q], c[kPacked ? 1 : Q], m[kPacked ? 1 : Q];
     unsigned int r0[kPacked ? Q : 1], r1[kPacked ? Q : 1];
+    // grouped modes: word 0 as loaded (r0 is overwritten while a request is retired), the key
+    // slope of the group the lane is in, and hosts found in that group (4 bits per request)
+    unsigned int r0_live[mode_is_grouped(MODE) ? Q : 1];
+    unsigned int group_slope = 0xFFFFFFFFu, group_found = 0u;
+    (void)r0_live; (void)group_slope; (void)group_found;
     KeyT t1[Q], t2[Q], t3[Q];
 #pragma unroll
     for (int q = 0; q < Q; ++q) {
@@ -276,6 +289,7 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
                 if (p.pack.fword[k]) w1 |= piece; else w0 |= piece;
             }
             r0[q] = w0; r1[q] = w1;
+            if (mode_is_grouped(MODE)) r0_live[q] = w0;
             g[q] = bad ? 0 : r.x;
         } else {
             if ((r.x | r.y | r.z | r.w) < 0) r.x = INT_MAX;  // a negative ask fits nowhere
@@ -343,13 +357,25 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
             const uint4 *R = reinterpret_cast<const uint4 *>(stage);
             const unsigned int guards0 = p.pack.guards, guards1 = p.pack.guards1;
             float cnt = 0.f, seen = 0.f;
+            (void)cnt; (void)seen;
             auto chunk = [&](auto width, int i0) {
                 constexpr int W = decltype(width)::value;
                 uint4 h[W];
 #pragma unroll
                 for (int u = 0; u < W; ++u) h[u] = R[i0 + u * L];
+                if constexpr (mode_is_grouped(MODE)) {
+                    // a new GPU-count group begins somewhere in this chunk: every request is live again
+                    // (the lane's hosts are in table order, so the last host of the chunk tells)
+                    const unsigned int slope = h[W - 1].w;
+                    if (slope != group_slope) {
+                        group_slope = slope;
+                        group_found = 0u;
+#pragma unroll
+                        for (int q = 0; q < Q; ++q) r0[q] = r0_live[q];
+                    }
+                }
                 bool hit;  // some pair of the chunk may enter its request's best three
-                if constexpr (mode_is_sorted(MODE)) {
+                if constexpr (mode_is_chained(MODE)) {
                     // table in key order: the capacity test alone decides (chained predicate)
                     hit = sorted_chunk_any_fit<Q, W, mode_two_masks(MODE)>(r0, r1, h, guards0, guards1);
                 } else {
@@ -374,7 +400,15 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
                             const bool bad = ((~d0 & guards0) | (~d1 & guards1)) != 0u;
                             const unsigned int key = mode_is_static(MODE) ? h[u].z : (unsigned int)g[q] * h[u].w + h[u].z;
                             insert3(t1[q], t2[q], t3[q], (KeyT)(bad ? 0xFFFFFFFFu : key));
+                            // hosts of the current group that fit this request, 4 bits per request
+                            if (mode_is_grouped(MODE) && !bad && h[u].w == group_slope) group_found += 1u << (4 * q);
                         }
+                    }
+                    if (mode_is_grouped(MODE)) {
+                        // three hosts of this group found: its later hosts all have larger keys
+#pragma unroll
+                        for (int q = 0; q < Q; ++q)
+                            if (((group_found >> (4 * q)) & 15u) >= 3u) r0[q] = guards0;
                     }
                     if (mode_is_sorted(MODE)) {
                         // three hosts found: every later host has a larger key. Retire the request
@@ -709,6 +743,8 @@ KernelFn pick_kernel(int mode, int L)
         case MODE_PACKED2_STATIC: return pick_kernel_l<MODE_PACKED2_STATIC>(L);
         case MODE_SORTED: return pick_kernel_l<MODE_SORTED>(L);
         case MODE_SORTED2: return pick_kernel_l<MODE_SORTED2>(L);
+        case MODE_GROUPED: return pick_kernel_l<MODE_GROUPED>(L);
+        case MODE_GROUPED2: return pick_kernel_l<MODE_GROUPED2>(L);
     }
     return nullptr;
 }
@@ -718,6 +754,7 @@ int snapshot_mode(const nbos_snapshot *s, int forced)
     if (s->key.key_bits == 64) return MODE_KEY64;
     if (forced == 1 || !s->pack.enabled) return MODE_PLAIN;
     const bool two = s->pack.guards != s->pack.guards1;
+    if (forced == 0 && s->key.grouped) return two ? MODE_GROUPED2 : MODE_GROUPED;
     if (forced == 2 || !s->key.static_key) return two ? MODE_PACKED2 : MODE_PACKED;
     if (forced == 3 || !s->presorted) return two ? MODE_PACKED2_STATIC : MODE_PACKED_STATIC;
     return two ? MODE_SORTED2 : MODE_SORTED;
@@ -786,7 +823,7 @@ int make_plan(const nbos_snapshot *s, long long total, long long batch, const nb
     int L = c.lanes_per_request;
     int blocks_per_sm = per_sm;
     {
-        const double pair_cost = mode_is_sorted(mode) ? 3.0 : mode_is_static(mode) ? 4.0 : mode_is_packed(mode) ? 5.0
+        const double pair_cost = mode_is_sorted(mode) ? 3.0 : mode_is_grouped(mode) ? 3.3 : mode_is_static(mode) ? 4.0 : mode_is_packed(mode) ? 5.0
                                  : mode == MODE_PLAIN ? 7.0 : 12.0;
         const double kPassCost = 490.0, kRequestCost = 190.0, kHostCost = 1.6, kMergeCost = 12.0;
         const double issue_rate[4] = {0.376, 0.472, 0.499, 0.529};  // per scheduler, by resident blocks

@@ -185,6 +185,54 @@ def test_packed_test_layouts_and_fallback(nb):
     assert_same(got, ref, "asks at the capacity maxima")
 
 
+def test_tables_grouped_by_gpu_count(nb):
+    """Hosts with different GPU counts (Section 3.4.1: 1 to 8 per server) rank differently for
+    different asks. With at most 8 distinct counts per snapshot the table is stored count by
+    count, each group in key order, and the kernel retires a request per group; with more counts
+    it falls back to computing the key for every pair. Same bytes as the checker either way."""
+    shapes = (dict(), dict(lanes_per_request=1), dict(lanes_per_request=4, requests_per_lane=2),
+              dict(lanes_per_request=32), dict(lanes_per_request=8, tile_hosts=32),
+              dict(lanes_per_request=2, host_split=3, tile_hosts=64))
+    # many hosts; tiny groups that several hosts of one chunk straddle; one ask dimension scarce
+    w_big = W.mixed_gpu_cluster(3000, 5000, seed=41)
+    w_tiny = W.mixed_gpu_cluster(40, 3000, seed=42)
+    w_scarce = W.mixed_gpu_cluster(1500, 4000, seed=43)
+    w_scarce.millicpus[0, :] = np.minimum(w_scarce.millicpus[0, :], 4000)   # most asks exceed it
+    w_two_masks = W.mixed_gpu_cluster(900, 3000, seed=44)
+    w_two_masks.mem_mb[0, 5] = 1 << 20
+    for w, packed in ((w_big, 1), (w_tiny, 1), (w_scarce, 1), (w_two_masks, 2)):
+        s = nb.snapshot_from_workload(w)
+        info = s.info()
+        assert (info.static_key, info.grouped, info.packed_test) == (0, 1, packed), w.name
+        nb.nbos_snapshot_destroy(s)
+        for key_order in (0, 1):
+            for flags in (0, 1):
+                for shape in shapes:
+                    got, ref = both(nb, w, key_order=key_order, flags=flags,
+                                    config=nb.launch_config(**shape) if shape else None)
+                    assert_same(got, ref, f"grouped {w.name} order={key_order} flags={flags} {shape}")
+    # several snapshots with different sets of GPU counts in one launch
+    parts = [W.mixed_gpu_cluster(500, 700, seed=50 + i) for i in range(3)]
+    parts[1].gpus_total[0, :] = np.where(parts[1].gpus_total[0, :] > 4, 8, 2)
+    parts[1].gpus_committed[0, :] = np.minimum(parts[1].gpus_committed[0, :], parts[1].gpus_total[0, :])
+    multi = dataclasses.replace(
+        parts[0], name="mixed_multi", n_snapshots=3,
+        **{k: np.concatenate([getattr(q, k) for q in parts], axis=0)
+           for k in W.Workload.HOST_FIELDS + ("limit_num", "limit_den", "requests")})
+    got, ref = both(nb, multi)
+    assert_same(got, ref, "grouped, three snapshots")
+    # more than 8 distinct GPU counts: not grouped
+    w_many = W.mixed_gpu_cluster(800, 3000, seed=45)
+    rng = np.random.Generator(np.random.PCG64(45))
+    w_many.gpus_total[0, :] = rng.integers(1, 13, size=800)
+    w_many.gpus_committed[0, :] = np.minimum(w_many.gpus_committed[0, :], w_many.gpus_total[0, :])
+    s = nb.snapshot_from_workload(w_many)
+    assert (s.info().static_key, s.info().grouped) == (0, 0)
+    nb.nbos_snapshot_destroy(s)
+    got, ref = both(nb, w_many)
+    assert_same(got, ref, "12 distinct GPU counts")
+
+
 def test_first_fit_variant(nb):
     """Stopping at the third feasible host (table in key order, same key slope everywhere) gives
     the same bytes as the full evaluation; where the conditions do not hold the flag is ignored."""
