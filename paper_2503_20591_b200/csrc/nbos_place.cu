@@ -66,7 +66,7 @@ __host__ __device__ constexpr int mode_record_bytes(int mode) { return mode == M
 __host__ __device__ constexpr int mode_max_q(int mode) { return mode == MODE_KEY64 ? 4 : 8; }
 // Resident blocks per SM the kernels are compiled for. The key-order modes touch their best-three
 // registers only on the rare update path, so 64 registers (a few spills there) buy a fourth block.
-__host__ __device__ constexpr int mode_blocks_per_sm(int mode) { return mode_is_sorted(mode) ? 4 : (mode_is_static(mode) || mode_is_grouped(mode)) ? 3 : 2; }
+__host__ __device__ constexpr int mode_blocks_per_sm(int mode) { return mode_is_chained(mode) ? 4 : mode_is_static(mode) ? 3 : 2; }
 constexpr int kStages = 3;
 
 struct PlaceParams {
@@ -263,35 +263,39 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
     // request registers: plain modes keep the four asks, packed modes the two packed words
     int g[Q], v[kPacked ? 1 : Q], c[kPacked ? 1 : Q], m[kPacked ? 1 : Q];
     unsigned int r0[kPacked ? Q : 1], r1[kPacked ? Q : 1];
-    // grouped modes: word 0 as loaded (r0 is overwritten while a request is retired), the key
-    // slope of the group the lane is in, and hosts found in that group (4 bits per request)
-    unsigned int r0_live[mode_is_grouped(MODE) ? Q : 1];
+    // grouped modes: the key slope of the group the lane is in, and hosts found in that group
+    // (4 bits per request)
     unsigned int group_slope = 0xFFFFFFFFu, group_found = 0u;
-    (void)r0_live; (void)group_slope; (void)group_found;
+    (void)group_slope; (void)group_found;
     KeyT t1[Q], t2[Q], t3[Q];
-#pragma unroll
-    for (int q = 0; q < Q; ++q) {
+    // request q of this lane, packed into the two words of the packed capacity test
+    auto load_packed = [&](int q, unsigned int &w0, unsigned int &w1, int &gpus) {
         const int idx = q * kGroups + grp;
         int4 r = make_int4(-1, 0, 0, 0);
         if (idx < count) r = __ldg(p.requests + first + idx);
-        if (kPacked) {
-            // an ask that is negative or larger than every host's capacity fits nowhere: encode it
-            // as a GPU ask above every host's gmax and keep the other fields inside their widths
-            const bool bad = ((r.x | r.y | r.z | r.w) < 0) | (r.x > p.pack.fmax[0]) | (r.y > p.pack.fmax[1]) |
-                             (r.z > p.pack.fmax[2]) | (r.w > p.pack.fmax[3]);
-            const unsigned int val[4] = {bad ? (unsigned int)p.pack.fmax[0] + 2u : (unsigned int)r.x + 1u,
-                                         bad ? 0u : (unsigned int)r.y, bad ? 0u : (unsigned int)r.z,
-                                         bad ? 0u : (unsigned int)r.w};
-            unsigned int w0 = 0u, w1 = 0u;
+        // an ask that is negative or larger than every host's capacity fits nowhere: encode it
+        // as a GPU ask above every host's gmax and keep the other fields inside their widths
+        const bool bad = ((r.x | r.y | r.z | r.w) < 0) | (r.x > p.pack.fmax[0]) | (r.y > p.pack.fmax[1]) |
+                         (r.z > p.pack.fmax[2]) | (r.w > p.pack.fmax[3]);
+        const unsigned int val[4] = {bad ? (unsigned int)p.pack.fmax[0] + 2u : (unsigned int)r.x + 1u,
+                                     bad ? 0u : (unsigned int)r.y, bad ? 0u : (unsigned int)r.z,
+                                     bad ? 0u : (unsigned int)r.w};
+        w0 = 0u; w1 = 0u;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const unsigned int piece = val[k] << p.pack.fshift[k];
-                if (p.pack.fword[k]) w1 |= piece; else w0 |= piece;
-            }
-            r0[q] = w0; r1[q] = w1;
-            if (mode_is_grouped(MODE)) r0_live[q] = w0;
-            g[q] = bad ? 0 : r.x;
+        for (int k = 0; k < 4; ++k) {
+            const unsigned int piece = val[k] << p.pack.fshift[k];
+            if (p.pack.fword[k]) w1 |= piece; else w0 |= piece;
+        }
+        gpus = bad ? 0 : r.x;
+    };
+#pragma unroll
+    for (int q = 0; q < Q; ++q) {
+        if (kPacked) {
+            load_packed(q, r0[q], r1[q], g[q]);
         } else {
+            const int idx = q * kGroups + grp;
+            int4 r = make_int4(-1, 0, 0, 0);
+            if (idx < count) r = __ldg(p.requests + first + idx);
             if ((r.x | r.y | r.z | r.w) < 0) r.x = INT_MAX;  // a negative ask fits nowhere
             g[q] = r.x; v[q] = r.y; c[q] = r.z; m[q] = r.w;
         }
@@ -370,8 +374,14 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
                     if (slope != group_slope) {
                         group_slope = slope;
                         group_found = 0u;
+                        // retired requests carry the guard mask in word 0: fetch the requests again
+                        // (a handful of times per pass; keeping a copy would cost 8 registers)
 #pragma unroll
-                        for (int q = 0; q < Q; ++q) r0[q] = r0_live[q];
+                        for (int q = 0; q < Q; ++q) {
+                            unsigned int w1_same;
+                            int gpus_same;
+                            load_packed(q, r0[q], w1_same, gpus_same);
+                        }
                     }
                 }
                 bool hit;  // some pair of the chunk may enter its request's best three
