@@ -864,6 +864,9 @@ int make_plan(const nbos_snapshot *s, long long total, long long batch, const nb
                         return kPassCost + qq * kRequestCost + per_host * (kHostCost + pair_cost * qq) + lg * qq * kMergeCost;
                     };
                     instr += (double)times * ((double)full * pass(max_q_kernel) + (rem ? pass(q) : 0.0));
+                    // a range that does not line up with the snapshots leaves some block a sliver of
+                    // another snapshot: one more pass over all hosts for a few requests
+                    if (part == 0 && total > B && (B % n_req != 0)) instr += pass(2);
                 }
                 const long long on_sm = (ctas + s->sm_count - 1) / s->sm_count;
                 const int resident = (int)(on_sm < j ? on_sm : j);
