@@ -120,6 +120,19 @@ int host_pipe(int device, HostPipe **out)
     return NBOS_OK;
 }
 
+}  // namespace
+
+int library_pool(int device, cudaMemPool_t *out)
+{
+    HostPipe *pipe = nullptr;
+    int rc = host_pipe(device, &pipe);
+    if (rc) return rc;
+    *out = pipe->pool;
+    return NBOS_OK;
+}
+
+namespace {
+
 nbos_snapshot *new_handle(const nbos_snapshot_desc *d)
 {
     nbos_snapshot *s = new (std::nothrow) nbos_snapshot();

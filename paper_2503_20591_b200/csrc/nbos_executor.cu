@@ -151,7 +151,10 @@ extern "C" int nbos_select_executors(const nbos_cluster_state *state, const int3
     const int H = state->n_hosts;
     char *packed = nullptr;  // stream-ordered temporary: 24 bytes per host
     const size_t fit_bytes = ((size_t)H * sizeof(int4) + 255) & ~(size_t)255;
-    cudaError_t e = cudaMallocAsync(reinterpret_cast<void **>(&packed), fit_bytes + (size_t)H * sizeof(int2), stream);
+    cudaMemPool_t pool = nullptr;
+    int rc = library_pool(device, &pool);
+    if (rc) return rc;
+    cudaError_t e = cudaMallocFromPoolAsync(reinterpret_cast<void **>(&packed), fit_bytes + (size_t)H * sizeof(int2), pool, stream);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return fail(NBOS_ERR_NO_MEMORY, "device allocation failed: %s", cudaGetErrorString(e));

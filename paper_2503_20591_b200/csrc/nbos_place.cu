@@ -987,7 +987,10 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
 
     if (K > 1) {
         const size_t cand_bytes = (size_t)K * (size_t)total * 3 * (k64 ? 8 : 4);
-        cudaError_t e = cudaMallocAsync(&p.cand, cand_bytes, stream);
+        cudaMemPool_t pool = nullptr;
+        rc = library_pool(s->device, &pool);
+        if (rc) return rc;
+        cudaError_t e = cudaMallocFromPoolAsync(&p.cand, cand_bytes, pool, stream);
         if (e != cudaSuccess) {
             cudaGetLastError();
             return fail(NBOS_ERR_NO_MEMORY, "could not allocate %zu bytes for slice candidates: %s", cand_bytes,
