@@ -759,6 +759,34 @@ KernelFn pick_kernel(int mode, int L)
     return nullptr;
 }
 
+// Resident blocks per SM of a placement kernel with `smem` bytes of dynamic shared memory, with
+// the kernel's shared-memory limit raised accordingly. Both runtime calls cost microseconds, which
+// is most of the host time of a small launch, so the answers are kept per (kernel, device, size).
+int kernel_occupancy(KernelFn fn, int device, size_t smem, int *per_sm)
+{
+    struct Entry { KernelFn fn; int device; size_t smem; int per_sm; };
+    static std::mutex mutex;
+    static Entry cache[256];
+    static int n_cached = 0;
+    std::lock_guard<std::mutex> lock(mutex);
+    for (int i = 0; i < n_cached; ++i)
+        if (cache[i].fn == fn && cache[i].device == device && cache[i].smem == smem) {
+            *per_sm = cache[i].per_sm;
+            return NBOS_OK;
+        }
+    NBOS_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    NBOS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(per_sm, fn, kThreads, smem));
+    // the attribute is per kernel: entries of the same kernel with a smaller size stay valid
+    // only while the limit is not lowered, so it is only ever raised
+    size_t largest = smem;
+    for (int i = 0; i < n_cached; ++i)
+        if (cache[i].fn == fn && cache[i].device == device && cache[i].smem > largest) largest = cache[i].smem;
+    if (largest > smem)
+        NBOS_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)largest));
+    if (n_cached < 256) cache[n_cached++] = Entry{fn, device, smem, *per_sm};
+    return NBOS_OK;
+}
+
 int snapshot_mode(const nbos_snapshot *s, int forced)
 {
     if (s->key.key_bits == 64) return MODE_KEY64;
@@ -817,9 +845,9 @@ int make_plan(const nbos_snapshot *s, long long total, long long batch, const nb
 
     KernelFn fn1 = pick_kernel(mode, 1);
     const size_t smem = (size_t)kStages * T * record + 2 * kStages * 8 + 16;
-    NBOS_CUDA_TRY(cudaFuncSetAttribute(fn1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 0;
-    NBOS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn1, kThreads, smem));
+    int rc_occ = kernel_occupancy(fn1, s->device, smem, &per_sm);
+    if (rc_occ) return rc_occ;
     if (per_sm < 1) return fail(NBOS_ERR_CUDA, "placement kernel does not fit on an SM (%zu bytes of shared memory)", smem);
 
     // Lanes per request and resident blocks per SM: for each choice, estimate the instructions a
@@ -963,8 +991,8 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
 
     KernelFn fn = pick_kernel(mode, L);
     if (!fn) return fail(NBOS_ERR_INVALID_ARG, "no kernel for this launch shape");
-    NBOS_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    NBOS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kThreads, smem));
+    rc = kernel_occupancy(fn, s->device, smem, &per_sm);
+    if (rc) return rc;
     if (per_sm < 1) return fail(NBOS_ERR_CUDA, "placement kernel does not fit on an SM (%zu bytes of shared memory)", smem);
 
     const int groups = kComputeThreads / L;
@@ -1085,9 +1113,9 @@ int launch_place_static(const nbos_snapshot *s, const int32_t *d_requests, int64
     const int L = 32;  // small batches are what this shape is for: one warp per request group
     KernelFn fn = pick_kernel(mode, L);
     const size_t smem = (size_t)kStages * T * record + 2 * kStages * 8 + 16;
-    NBOS_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     int per_sm = 0;
-    NBOS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, kThreads, smem));
+    rc = kernel_occupancy(fn, device, smem, &per_sm);
+    if (rc) return rc;
     if (per_sm < 1) return fail(NBOS_ERR_CUDA, "placement kernel does not fit on an SM");
     const int groups = kComputeThreads / L;
     long long req_ctas = (total + groups - 1) / groups;
