@@ -238,7 +238,7 @@ int nbos_place_batch_ex(const nbos_snapshot *snap, const int32_t *requests,
 
 /*
  * Same operation with HOST buffers (pinned memory makes the copies asynchronous and faster, but
- * any host memory works). The batch is cut into up to 16 chunks whose host-to-device copy, kernel
+ * any host memory works). The batch is cut into up to 8 chunks whose host-to-device copy, kernel
  * and device-to-host copy overlap on three internal streams (created once per device; calls on
  * the same device take turns). Device staging comes from the library's own memory pool. Returns
  * after the results are in the host buffers.
