@@ -276,7 +276,7 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
 // keys are unique, so the position of host i is the number of hosts with a smaller key. Each
 // block counts, for 256 hosts, the smaller keys inside one chunk of kRankChunk keys staged in
 // shared memory, and adds its partial count to rank[i]. grid (ceil(Hpad/256), ceil(Hpad/chunk), N).
-constexpr int kRankChunk = 1024;
+constexpr int kRankChunk = 256;
 __global__ void __launch_bounds__(256) rank_kernel(const unsigned long long *sortkey, unsigned int *rank, int Hpad)
 {
     __shared__ unsigned long long chunk[kRankChunk];
