@@ -64,9 +64,11 @@ __host__ __device__ constexpr bool mode_is_static(int mode) { return mode == MOD
 __host__ __device__ constexpr bool mode_two_masks(int mode) { return mode == MODE_PACKED2 || mode == MODE_PACKED2_STATIC || mode == MODE_SORTED2 || mode == MODE_GROUPED2; }
 __host__ __device__ constexpr int mode_record_bytes(int mode) { return mode == MODE_KEY64 ? 32 : mode == MODE_PLAIN ? 24 : 16; }
 __host__ __device__ constexpr int mode_max_q(int mode) { return mode == MODE_KEY64 ? 4 : 8; }
-// Resident blocks per SM the kernels are compiled for. The key-order modes touch their best-three
-// registers only on the rare update path, so 64 registers (a few spills there) buy a fourth block.
-__host__ __device__ constexpr int mode_blocks_per_sm(int mode) { return mode_is_chained(mode) ? 4 : mode_is_static(mode) ? 3 : 2; }
+// Resident blocks per SM the kernels are compiled for. The modes that rank hosts by their own key
+// touch most best-three registers only on the rare update path, so 64 registers (a few spills
+// there) buy a fourth block; with the key computed per pair the same limit spills in the loop
+// (measured slower), so those modes stay at two blocks.
+__host__ __device__ constexpr int mode_blocks_per_sm(int mode) { return (mode_is_chained(mode) || mode_is_static(mode)) ? 4 : 2; }
 constexpr int kStages = 3;
 
 struct PlaceParams {
