@@ -35,7 +35,7 @@ ALGORITHMIC_OPS_PER_PAIR = 6      # 4 capacity compares + 1 multiply-add (key) +
 L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (read + write) of one placement-kernel launch on the default workload, from the ncu
 # capture summarised under profiles/. None while no capture matches the current kernel.
-PLACE_KERNEL_DRAM_BYTES_PER_LAUNCH = 16_942_848
+PLACE_KERNEL_DRAM_BYTES_PER_LAUNCH = 16_937_984
 # Warp instructions the placement kernel executes per 32 pairs on the default workload, from the
 # same capture (smsp__inst_executed.sum / (pairs / 32)).
 PLACE_KERNEL_WARP_INSTR_PER_32_PAIRS = 3.59
