@@ -12,7 +12,7 @@ CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libnbos.so")
 SOURCES = ("nbos_api.cu", "nbos_derive.cu", "nbos_place.cu", "nbos_executor.cu", "nbos_cluster.cu", "nbos_sequential.cu", "nbos_probe.cu")
 HEADERS = (os.path.join(ROOT, "include", "nbos.h"), os.path.join(ROOT, "include", "nbos_probe.h"),
-           os.path.join(CSRC, "nbos_internal.h"), os.path.join(CSRC, "nbos_ptx.cuh"), os.path.join(CSRC, "nbos_sorted_chunk.cuh"))
+           os.path.join(CSRC, "nbos_internal.h"), os.path.join(CSRC, "nbos_ptx.cuh"), os.path.join(CSRC, "nbos_sorted_chunk.cuh"), os.path.join(CSRC, "nbos_ranked_chunk.cuh"))
 ARCH_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 

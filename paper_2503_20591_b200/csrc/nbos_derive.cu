@@ -301,8 +301,10 @@ struct FinalizeArgs {
     int4 *feas;
     void *ab;
     uint4 *pk;
+    uint2 *rk;
     int Hpad;
     PackLayout pack;
+    RankLayout ranked;
 };
 
 // grid (ceil(Hpad / 256), N): move the records into visiting order and build the packed form.
@@ -324,6 +326,16 @@ __global__ void __launch_bounds__(256) finalize_kernel(const FinalizeArgs a)
 #pragma unroll
         for (int c = 0; c < 4; ++c) w[a.pack.fword[c]] |= cap[c] << a.pack.fshift[c];
         a.pk[base + j] = make_uint4(w[0], w[1], (unsigned int)p.x, (unsigned int)p.y);
+    }
+    if (a.ranked.enabled) {
+        // ranked form: coarse capacities and the host's position in key order, two words
+        const unsigned int cap[4] = {(unsigned int)(f.x + 1), (unsigned int)f.y, (unsigned int)f.z,
+                                     (unsigned int)f.w};
+        unsigned int w[2] = {a.ranked.guards, a.ranked.guards};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) w[a.ranked.fword[c]] |= (cap[c] >> a.ranked.fdrop[c]) << a.ranked.fshift[c];
+        w[a.ranked.fword[4]] |= (a.ranked.rank_top - j) << a.ranked.fshift[4];
+        a.rk[base + j] = make_uint2(w[0], w[1]);
     }
 }
 
@@ -363,6 +375,7 @@ Layout workspace_layout(int N, int Hpad)
     l.off_feas = o;    o = up(o + (size_t)N * Hpad * sizeof(int4));
     l.off_ab = o;      o = up(o + (size_t)N * Hpad * sizeof(ulonglong2));
     l.off_pk = o;      o = up(o + (size_t)N * Hpad * sizeof(uint4));
+    l.off_rk = o;      o = up(o + (size_t)N * Hpad * sizeof(uint2));
     l.off_tmp_feas = o; o = up(o + (size_t)N * Hpad * sizeof(int4));
     l.off_tmp_ab = o;  o = up(o + (size_t)N * Hpad * sizeof(ulonglong2));
     l.off_tmp_seq = o; o = up(o + (size_t)N * Hpad * sizeof(int4));
@@ -456,7 +469,8 @@ int emit_tables(DeriveCtx &c)
     if (s->presorted)
         rank_kernel<<<dim3((Hpad + 255) / 256, (Hpad + kRankChunk - 1) / kRankChunk, N), 256, 0, c.stream>>>(sortkey, perm, Hpad);
     FinalizeArgs fa{tmp_feas, tmp_ab, s->presorted ? perm : nullptr, reinterpret_cast<int4 *>(c.ws + c.lay.off_feas),
-                    c.ws + c.lay.off_ab, reinterpret_cast<uint4 *>(c.ws + c.lay.off_pk), Hpad, s->pack};
+                    c.ws + c.lay.off_ab, reinterpret_cast<uint4 *>(c.ws + c.lay.off_pk),
+                    reinterpret_cast<uint2 *>(c.ws + c.lay.off_rk), Hpad, s->pack, s->rank};
     if (k.key_bits == 32)
         finalize_kernel<uint2><<<grid, 256, 0, c.stream>>>(fa);
     else
@@ -571,12 +585,20 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     idle_max = (int)((1u << k.bits_idle) - 1u);
     s->idle_max = idle_max;
 
+    // field widths of the four capacity components, from the scanned maxima
+    int width[4];
+    width[0] = bits_for((unsigned long long)fmax[0] + 2);  // stored +1, and one more for "fits nowhere"
+    for (int c2 = 1; c2 < 4; ++c2) width[c2] = fmax[c2] ? bits_for((unsigned long long)fmax[c2]) : 1;
+    // largest value each field can take (not merely the largest present now): asks up to it are
+    // compared exactly, and a later update may raise capacities up to it
+    int field_max[4];
+    field_max[0] = (int)((1u << width[0]) - 3u);
+    for (int c2 = 1; c2 < 4; ++c2) field_max[c2] = (int)((1u << width[c2]) - 1u);
+
     // packed capacity test: the two widest components become the high fields of the two words
     PackLayout pk = {};
     if (k.key_bits == 32) {
-        int width[4], order[4] = {0, 1, 2, 3};
-        width[0] = bits_for((unsigned long long)fmax[0] + 2);  // stored +1, and one more for "fits nowhere"
-        for (int c2 = 1; c2 < 4; ++c2) width[c2] = fmax[c2] ? bits_for((unsigned long long)fmax[c2]) : 1;
+        int order[4] = {0, 1, 2, 3};
         for (int i = 0; i < 4; ++i)
             for (int j = i + 1; j < 4; ++j)
                 if (width[order[j]] > width[order[i]]) { int t = order[i]; order[i] = order[j]; order[j] = t; }
@@ -589,10 +611,7 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
             pk.enabled = 1;
             pk.guards = 0x80000000u | (1u << lo_a);
             pk.guards1 = 0x80000000u | (1u << lo_b);
-            // largest value each field can take (not merely the largest present now): asks up to it
-            // are compared exactly, and a later update may raise capacities up to it
-            pk.fmax[0] = (int)((1u << width[0]) - 3u);
-            for (int c2 = 1; c2 < 4; ++c2) pk.fmax[c2] = (int)((1u << width[c2]) - 1u);
+            for (int c2 = 0; c2 < 4; ++c2) pk.fmax[c2] = field_max[c2];
             pk.fword[order[0]] = 0; pk.fshift[order[0]] = lo_a + 1;
             pk.fword[order[3]] = 0; pk.fshift[order[3]] = 0;
             pk.fword[order[1]] = 1; pk.fshift[order[1]] = lo_b + 1;
@@ -601,6 +620,55 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     }
     s->pack = pk;
     s->presorted = Hpad <= kSortMaxHosts;
+
+    // Ranked form (see RankLayout): six slots -- three per word at the same bit positions -- for
+    // the four capacities, the rank and one unused slot. Components are paired by width (the two
+    // narrowest share the lowest slot, and so on); a slot is as wide as its wider member, and
+    // while the three widths exceed the 29 bits left beside the guards the widest slot that may
+    // shrink does: the GPU component and the rank stay exact, the others lose low bits.
+    RankLayout rl = {};
+    if (k.key_bits == 32 && k.static_key && s->presorted) {
+        int w6[6] = {width[0], width[1], width[2], width[3], bits_for((unsigned long long)(Hpad - 1)), 0};
+        int order[6] = {0, 1, 2, 3, 4, 5};
+        for (int i = 0; i < 6; ++i)
+            for (int j = i + 1; j < 6; ++j)
+                if (w6[order[j]] < w6[order[i]]) { int t = order[i]; order[i] = order[j]; order[j] = t; }
+        int slot_w[3], slot_min[3];
+        for (int sl = 0; sl < 3; ++sl) {
+            const int a = order[2 * sl], b = order[2 * sl + 1];
+            slot_w[sl] = w6[a] > w6[b] ? w6[a] : w6[b];
+            slot_min[sl] = 1;
+            if ((a == 0 || a == 4) && w6[a] > slot_min[sl]) slot_min[sl] = w6[a];
+            if ((b == 0 || b == 4) && w6[b] > slot_min[sl]) slot_min[sl] = w6[b];
+            if (slot_w[sl] < slot_min[sl]) slot_w[sl] = slot_min[sl];
+        }
+        bool fits = true;
+        while (slot_w[0] + slot_w[1] + slot_w[2] > 29) {
+            int pick = -1;
+            for (int sl = 0; sl < 3; ++sl)
+                if (slot_w[sl] > slot_min[sl] && (pick < 0 || slot_w[sl] > slot_w[pick])) pick = sl;
+            if (pick < 0) { fits = false; break; }
+            --slot_w[pick];
+        }
+        if (fits) {
+            slot_w[2] = 29 - slot_w[0] - slot_w[1];  // the top slot takes what is left
+            const int slot_shift[3] = {0, slot_w[0] + 1, slot_w[0] + slot_w[1] + 2};
+            rl.enabled = 1;
+            rl.guards = 0x80000000u | (1u << slot_w[0]) | (1u << (slot_w[0] + slot_w[1] + 1));
+            for (int sl = 0; sl < 3; ++sl)
+                for (int half = 0; half < 2; ++half) {
+                    const int comp = order[2 * sl + half];
+                    if (comp == 5) continue;  // the unused slot: host field 0 against request field 0
+                    rl.fword[comp] = half;
+                    rl.fshift[comp] = slot_shift[sl];
+                    rl.fdrop[comp] = w6[comp] > slot_w[sl] ? w6[comp] - slot_w[sl] : 0;
+                }
+            for (int c2 = 0; c2 < 4; ++c2) rl.fmax[c2] = field_max[c2];
+            rl.rank_top = (unsigned int)(Hpad - 1);
+            rl.rank_mask = ((1u << w6[4]) - 1u) << rl.fshift[4];
+        }
+    }
+    s->rank = rl;
     // Hosts with different GPU counts rank differently for different asks, but within one GPU
     // count the order is the same for every ask. With few distinct counts the table is stored
     // count by count, each group in key order, and the placement kernel treats every group like
@@ -619,6 +687,7 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     s->d_feas = reinterpret_cast<const int4 *>(c.ws + c.lay.off_feas);
     s->d_ab = c.ws + c.lay.off_ab;
     s->d_pk = reinterpret_cast<const uint4 *>(c.ws + c.lay.off_pk);
+    s->d_rk = reinterpret_cast<const uint2 *>(c.ws + c.lay.off_rk);
     s->d_host_feas = reinterpret_cast<const int4 *>(c.ws + c.lay.off_tmp_feas);
     s->d_host_ab = c.ws + c.lay.off_tmp_ab;
     s->d_host_seq = reinterpret_cast<const int4 *>(c.ws + c.lay.off_tmp_seq);
@@ -635,13 +704,15 @@ int update_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     DeriveCtx c = make_ctx(s, d_G, d_S, d_C, d_AV, d_AC, d_AM, stream);
     int rc = stage_limits(c, d);
     if (rc) return rc;
+    const int *fm = s->pack.enabled ? s->pack.fmax : s->rank.fmax;  // the same values in both layouts
     ScanArgs sa{d_G, d_S, d_C, d_AV, d_AC, d_AM, c.limits_arg, c.limit0,
                 reinterpret_cast<SnapStats *>(c.ws + c.lay.off_stats), s->H, s->R, s->flags,
                 s->d_status,
                 s->key.static_key ? nullptr : reinterpret_cast<const long long *>(c.ws + c.lay.off_lambda),
                 reinterpret_cast<const int *>(c.ws + c.lay.off_g_single),
-                s->key.bits_sr >= 64 ? ~0ull : ((1ull << s->key.bits_sr) - 1ull), s->idle_max, s->pack.enabled,
-                {s->pack.fmax[0], s->pack.fmax[1], s->pack.fmax[2], s->pack.fmax[3]}};
+                s->key.bits_sr >= 64 ? ~0ull : ((1ull << s->key.bits_sr) - 1ull), s->idle_max,
+                s->pack.enabled || s->rank.enabled,
+                {fm[0], fm[1], fm[2], fm[3]}};
     scan_kernel<<<dim3(c.bx, s->N), 256, 0, stream>>>(sa);
     NBOS_CUDA_TRY(cudaGetLastError());
     return emit_tables(c);

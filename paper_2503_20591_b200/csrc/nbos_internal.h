@@ -42,7 +42,7 @@ enum : unsigned int {
 };
 
 struct Layout {
-    size_t off_status, off_limits, off_sums, off_stats, off_lambda, off_g_single, off_feas, off_ab, off_pk;
+    size_t off_status, off_limits, off_sums, off_stats, off_lambda, off_g_single, off_feas, off_ab, off_pk, off_rk;
     size_t off_tmp_feas, off_tmp_ab, off_tmp_seq, off_sortkey, off_perm, total;
 };
 Layout workspace_layout(int n_snapshots, int hosts_padded);
@@ -70,6 +70,30 @@ struct PackLayout {
     unsigned int guards1;   // guard bits of word 1 (equal to `guards` when the layouts coincide)
 };
 
+// One-subtraction encoding of the whole pair step for snapshots whose hosts rank the same for
+// every ask (static key) and whose table is stored in key order. A host is a pair of 32-bit words
+// (one 64-bit value); each word has three fields at the same bit positions in both words, every
+// field with a guard bit right above it (the top one at bit 31). Five of the six fields are used:
+// the four capacities of Section 3.2.1 (component 0 stored as gmax + 1 against ask + 1) and the
+// host's rank in the order of Section 3.4.1, stored as rank_top - position against the request's
+// rank_top + 1 - (position of its current third best), so that the guard survives exactly when
+// the host ranks before the third best. host - request (one 64-bit subtraction, or two 32-bit
+// ones) keeps every guard set exactly when the host fits the ask in all four resources and would
+// enter the request's best three. Capacities wider than their field lose their low `fdrop` bits
+// on both sides: floor(ask / 2^d) <= floor(capacity / 2^d) whenever ask <= capacity, so the coarse
+// test never rejects a feasible host; pairs that pass it are re-tested exactly before the best
+// three change. The GPU component and the rank are always exact.
+struct RankLayout {
+    int enabled;
+    int fmax[4];     // largest ask that any host could satisfy, per component (as PackLayout::fmax)
+    int fword[5];    // word (0 / 1) of components 0..3 and of the rank (index 4)
+    int fshift[5];   // bit position inside that word
+    int fdrop[5];    // low bits dropped before the component is stored (0 = exact)
+    unsigned int guards;    // guard bits, the same in both words
+    unsigned int rank_top;  // host field = rank_top - position in the table
+    unsigned int rank_mask; // bits of the rank field inside its word
+};
+
 }  // namespace nbos
 
 struct nbos_snapshot {
@@ -84,6 +108,8 @@ struct nbos_snapshot {
     const void *d_ab;     // [N][Hpad] uint2 (32-bit keys) or ulonglong2 (64-bit keys): (A, B)
     const uint4 *d_pk;    // [N][Hpad] (word0, word1, A, B), only when pack.enabled
     nbos::PackLayout pack;
+    const uint2 *d_rk;    // [N][Hpad] (word0, word1) of the ranked form, only when rank.enabled
+    nbos::RankLayout rank;
     int presorted;
     int idle_max;             // the key's idle field stores idle_max - (G - C)
     // the same records in host-index order (what the derivation staged), for sequential placement

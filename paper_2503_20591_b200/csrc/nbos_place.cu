@@ -27,6 +27,7 @@
 
 #include "nbos_internal.h"
 #include "nbos_ptx.cuh"
+#include "nbos_ranked_chunk.cuh"
 #include "nbos_sorted_chunk.cuh"
 
 namespace nbos {
@@ -53,29 +54,35 @@ enum : int {
                              // key order (a request is retired for the rest of a group once it has three
                              // hosts of that group), keys are computed only for the hosts that fit
     MODE_GROUPED2 = 9,       // as 8 with two guard masks
-    MODE_COUNT = 10,
+    MODE_RANKED = 10,        // static key, table in key order: capacities and rank in one 64-bit value per
+                             // host and per request, one subtraction + one logic operation per pair;
+                             // pairs that pass are re-tested exactly          (records: rk, then feas + ab)
+    MODE_COUNT = 11,
 };
-__host__ __device__ constexpr bool mode_is_packed(int mode) { return mode >= MODE_PACKED; }
+__host__ __device__ constexpr bool mode_is_ranked(int mode) { return mode == MODE_RANKED; }
+__host__ __device__ constexpr bool mode_is_packed(int mode) { return mode >= MODE_PACKED && mode <= MODE_GROUPED2; }
 __host__ __device__ constexpr bool mode_is_sorted(int mode) { return mode == MODE_SORTED || mode == MODE_SORTED2; }
 __host__ __device__ constexpr bool mode_is_grouped(int mode) { return mode == MODE_GROUPED || mode == MODE_GROUPED2; }
 // modes whose pair step is the capacity test alone (chained predicate, no key work per pair)
 __host__ __device__ constexpr bool mode_is_chained(int mode) { return mode_is_sorted(mode) || mode_is_grouped(mode); }
 __host__ __device__ constexpr bool mode_is_static(int mode) { return mode == MODE_PACKED_STATIC || mode == MODE_PACKED2_STATIC || mode_is_sorted(mode); }
 __host__ __device__ constexpr bool mode_two_masks(int mode) { return mode == MODE_PACKED2 || mode == MODE_PACKED2_STATIC || mode == MODE_SORTED2 || mode == MODE_GROUPED2; }
-__host__ __device__ constexpr int mode_record_bytes(int mode) { return mode == MODE_KEY64 ? 32 : mode == MODE_PLAIN ? 24 : 16; }
+__host__ __device__ constexpr int mode_record_bytes(int mode) { return mode == MODE_KEY64 ? 32 : mode == MODE_PLAIN ? 24 : mode == MODE_RANKED ? 8 : 16; }
 __host__ __device__ constexpr int mode_max_q(int mode) { return mode == MODE_KEY64 ? 4 : 8; }
 // Resident blocks per SM the kernels are compiled for. The modes that rank hosts by their own key
 // touch most best-three registers only on the rare update path, so 64 registers (a few spills
 // there) buy a fourth block; with the key computed per pair the same limit spills in the loop
 // (measured slower), so those modes stay at two blocks.
-__host__ __device__ constexpr int mode_blocks_per_sm(int mode) { return (mode_is_chained(mode) || mode_is_static(mode)) ? 4 : 2; }
+__host__ __device__ constexpr int mode_blocks_per_sm(int mode) { return (mode_is_chained(mode) || mode_is_static(mode) || mode_is_ranked(mode)) ? 4 : 2; }
 constexpr int kStages = 3;
 
 struct PlaceParams {
     const int4 *feas;       // [N][Hpad]
     const void *ab;         // [N][Hpad] pairs (A, B)
     const uint4 *pk;        // [N][Hpad] (word0, word1, A, B), packed modes
+    const uint2 *rk;        // [N][Hpad] (word0, word1), ranked mode
     PackLayout pack;
+    RankLayout rank;
     const int4 *requests;   // [N * B]
     int32_t *out_hosts;     // [N * B * 3]
     int32_t *out_found;     // [N * B] or null
@@ -475,6 +482,149 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
     return true;
 }
 
+// ---- one pass in ranked form ------------------------------------------------------------------
+// Same contract as run_pass. The best three of a request are kept as positions in the table
+// (which is stored in key order, so a smaller position is a smaller key) and turned into keys
+// after the last tile. Per pair: ranked_chunk_any_pass. When a chunk reports a pass, its pairs
+// are re-tested with the exact records (four compares against the request as it was given),
+// fitting hosts enter the best three, and the request's rank field is set from its new third
+// best.
+template <int Q, int L>
+__device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned char *stages,
+                                                uint32_t stage_bytes, uint32_t full_bar,
+                                                uint32_t empty_bar, volatile unsigned int *abort_flag,
+                                                uint32_t &ring_pos, int tile_begin, int tile_end,
+                                                int slice, long long first, int count, int n)
+{
+    constexpr unsigned int kNone = 0xFFFFFFFFu;
+    constexpr int kGroups = kComputeThreads / L;
+    const int tid = threadIdx.x;
+    const int sub = tid % L;
+    const int grp = tid / L;
+    const int lane = tid & 31;
+    const size_t row = (size_t)n * p.Hpad;
+    const unsigned int guards = p.rank.guards;
+    const int rank_shift = p.rank.fshift[4] + 32 * p.rank.fword[4];
+    const unsigned long long rank_mask = (unsigned long long)p.rank.rank_mask << (32 * p.rank.fword[4]);
+
+    // the ask as given, with a GPU count no host has when it fits nowhere (negative field)
+    auto load_request = [&](int q) -> int4 {
+        const int idx = q * kGroups + grp;
+        int4 r = make_int4(-1, 0, 0, 0);
+        if (idx < count) r = __ldg(p.requests + first + idx);
+        if ((r.x | r.y | r.z | r.w) < 0) r.x = INT_MAX;
+        return r;
+    };
+
+    unsigned long long rq[Q];
+    unsigned int t1[Q], t2[Q], t3[Q];
+#pragma unroll
+    for (int q = 0; q < Q; ++q) {
+        const int4 r = load_request(q);
+        // an ask above every host's capacity in some resource fits nowhere either: encode both
+        // cases as a GPU ask above every gmax and keep the other fields inside their widths
+        const bool bad = (r.x > p.rank.fmax[0]) | (r.y > p.rank.fmax[1]) | (r.z > p.rank.fmax[2]) |
+                         (r.w > p.rank.fmax[3]);
+        const unsigned int val[4] = {bad ? (unsigned int)p.rank.fmax[0] + 2u : (unsigned int)r.x + 1u,
+                                     bad ? 0u : (unsigned int)r.y, bad ? 0u : (unsigned int)r.z,
+                                     bad ? 0u : (unsigned int)r.w};
+        unsigned int w0 = 0u, w1 = 0u;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const unsigned int piece = (val[k] >> p.rank.fdrop[k]) << p.rank.fshift[k];
+            if (p.rank.fword[k]) w1 |= piece; else w0 |= piece;
+        }
+        rq[q] = (unsigned long long)w0 | ((unsigned long long)w1 << 32);  // rank field 0: every rank passes
+        t1[q] = kNone; t2[q] = kNone; t3[q] = kNone;
+    }
+
+    const int T = p.tile_hosts;
+    for (int t = tile_begin; t < tile_end; ++t, ++ring_pos) {
+        const uint32_t s = ring_pos % kStages;
+        const uint32_t parity = (ring_pos / kStages) & 1u;
+        if (!mbar_wait(full_bar + 8u * s, parity, abort_flag)) return false;
+        const unsigned long long *R = reinterpret_cast<const unsigned long long *>(stages + (size_t)s * stage_bytes);
+        const int pos0 = t * T;
+        int hosts = p.Hpad - pos0;
+        if (hosts > T) hosts = T;
+        auto chunk = [&](auto width, int i0) {
+            constexpr int W = decltype(width)::value;
+            unsigned long long h[W];
+            if constexpr (L == 1 && W == 4) {
+                // consecutive hosts: two 128-bit shared-memory loads (i0 is a multiple of 4)
+                const ulonglong2 a = *reinterpret_cast<const ulonglong2 *>(R + i0);
+                const ulonglong2 b = *reinterpret_cast<const ulonglong2 *>(R + i0 + 2);
+                h[0] = a.x; h[1] = a.y; h[2] = b.x; h[3] = b.y;
+            } else {
+#pragma unroll
+                for (int u = 0; u < W; ++u) h[u] = R[i0 + u * L];
+            }
+            if (ranked_chunk_any_pass<Q, W>(rq, h, guards)) {
+                // rare: exact re-test of the chunk's pairs, then the new thresholds
+                int4 f[W];
+#pragma unroll
+                for (int u = 0; u < W; ++u) f[u] = __ldg(p.feas + row + pos0 + i0 + u * L);
+#pragma unroll
+                for (int q = 0; q < Q; ++q) {
+                    const int4 r = load_request(q);
+#pragma unroll
+                    for (int u = 0; u < W; ++u) {
+                        const bool ok = (r.x <= f[u].x) & (r.y <= f[u].y) & (r.z <= f[u].z) & (r.w <= f[u].w);
+                        insert3(t1[q], t2[q], t3[q], ok ? (unsigned int)(pos0 + i0 + u * L) : kNone);
+                    }
+                    const unsigned int field = t3[q] == kNone ? 0u : p.rank.rank_top + 1u - t3[q];
+                    rq[q] = (rq[q] & ~rank_mask) | ((unsigned long long)field << rank_shift);
+                }
+            }
+        };
+        int i = sub;
+        for (; i + 3 * L < hosts; i += 4 * L) chunk(std::integral_constant<int, 4>{}, i);
+        for (; i < hosts; i += L) chunk(std::integral_constant<int, 1>{}, i);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_bar + 8u * s);
+    }
+
+    // merge the L lanes of a group (positions are unique)
+#pragma unroll
+    for (int mask = 1; mask < L; mask <<= 1) {
+#pragma unroll
+        for (int q = 0; q < Q; ++q) {
+            const unsigned int o1 = __shfl_xor_sync(0xFFFFFFFFu, t1[q], mask);
+            const unsigned int o2 = __shfl_xor_sync(0xFFFFFFFFu, t2[q], mask);
+            const unsigned int o3 = __shfl_xor_sync(0xFFFFFFFFu, t3[q], mask);
+            insert3(t1[q], t2[q], t3[q], o1);
+            insert3(t1[q], t2[q], t3[q], o2);
+            insert3(t1[q], t2[q], t3[q], o3);
+        }
+    }
+
+    if (sub == 0) {
+        const uint2 *AB = reinterpret_cast<const uint2 *>(p.ab) + row;
+#pragma unroll
+        for (int q = 0; q < Q; ++q) {
+            const int idx = q * kGroups + grp;
+            if (idx >= count) continue;
+            const long long r = first + idx;
+            // position -> key (its low bits are the host id; all hosts share the key slope, so
+            // the intercepts order like the keys)
+            const unsigned int k1 = t1[q] == kNone ? kNone : __ldg(&AB[t1[q]].x);
+            const unsigned int k2 = t2[q] == kNone ? kNone : __ldg(&AB[t2[q]].x);
+            const unsigned int k3 = t3[q] == kNone ? kNone : __ldg(&AB[t3[q]].x);
+            if (p.K > 1) {
+                unsigned int *cand = reinterpret_cast<unsigned int *>(p.cand) + ((long long)slice * p.n_req + (r - p.first_req)) * 3;
+                cand[0] = k1; cand[1] = k2; cand[2] = k3;
+            } else {
+                int32_t *o = p.out_hosts + r * 3;
+                o[0] = k1 == kNone ? -1 : (int)(k1 & p.id_mask);
+                o[1] = k2 == kNone ? -1 : (int)(k2 & p.id_mask);
+                o[2] = k3 == kNone ? -1 : (int)(k3 & p.id_mask);
+                if (p.out_found) p.out_found[r] = (k1 != kNone) + (k2 != kNone) + (k3 != kNone);
+            }
+        }
+    }
+    return true;
+}
+
 template <int L, int MODE>
 __global__ void __launch_bounds__(kThreads, mode_blocks_per_sm(MODE))
 place_kernel(const __grid_constant__ PlaceParams p)
@@ -534,7 +684,11 @@ place_kernel(const __grid_constant__ PlaceParams p)
                 int hosts = p.Hpad - t * T;
                 if (hosts > T) hosts = T;
                 const uint32_t dst = stage0 + s * stage_bytes;
-                if (kPacked) {
+                if (mode_is_ranked(MODE)) {
+                    const uint32_t bytes = (uint32_t)hosts * 8u;
+                    mbar_arrive_expect_tx(full_bar + 8u * s, bytes);
+                    bulk_copy_g2s(dst, p.rk + row + (size_t)t * T, bytes, full_bar + 8u * s);
+                } else if (kPacked) {
                     const uint32_t bytes = (uint32_t)hosts * 16u;
                     mbar_arrive_expect_tx(full_bar + 8u * s, bytes);
                     bulk_copy_g2s(dst, p.pk + row + (size_t)t * T, bytes, full_bar + 8u * s);
@@ -569,13 +723,17 @@ place_kernel(const __grid_constant__ PlaceParams p)
     uint32_t ring_pos = 0;
     bool ok = true;
     while (ok && passes.next(n, first, count, q)) {
-#define NBOS_PASS(QV)                                                                         \
-    ok = run_pass<QV, L, MODE>(p, smem, stage_bytes, full_bar, empty_bar, abort_flag, ring_pos, \
-                               tile_begin, tile_end, slice, first, count)
-        if (MAXQ >= 8 && q == 8) NBOS_PASS(8);
-        else if (MAXQ >= 4 && q == 4) NBOS_PASS(4);
-        else if (MAXQ >= 2 && q == 2) NBOS_PASS(2);
-        else NBOS_PASS(1);
+#define NBOS_PASS(QV)                                                                                 \
+    if constexpr (mode_is_ranked(MODE))                                                               \
+        ok = run_pass_ranked<QV, L>(p, smem, stage_bytes, full_bar, empty_bar, abort_flag, ring_pos,  \
+                                    tile_begin, tile_end, slice, first, count, n);                    \
+    else                                                                                              \
+        ok = run_pass<QV, L, MODE>(p, smem, stage_bytes, full_bar, empty_bar, abort_flag, ring_pos,   \
+                                   tile_begin, tile_end, slice, first, count)
+        if (MAXQ >= 8 && q == 8) { NBOS_PASS(8); }
+        else if (MAXQ >= 4 && q == 4) { NBOS_PASS(4); }
+        else if (MAXQ >= 2 && q == 2) { NBOS_PASS(2); }
+        else { NBOS_PASS(1); }
 #undef NBOS_PASS
     }
     if (!ok) atomicOr(p.status, 1u);
@@ -757,6 +915,7 @@ KernelFn pick_kernel(int mode, int L)
         case MODE_SORTED2: return pick_kernel_l<MODE_SORTED2>(L);
         case MODE_GROUPED: return pick_kernel_l<MODE_GROUPED>(L);
         case MODE_GROUPED2: return pick_kernel_l<MODE_GROUPED2>(L);
+        case MODE_RANKED: return pick_kernel_l<MODE_RANKED>(L);
     }
     return nullptr;
 }
@@ -792,9 +951,10 @@ int kernel_occupancy(KernelFn fn, int device, size_t smem, int *per_sm)
 int snapshot_mode(const nbos_snapshot *s, int forced)
 {
     if (s->key.key_bits == 64) return MODE_KEY64;
+    if (forced == 0 && s->rank.enabled) return MODE_RANKED;
     if (forced == 1 || !s->pack.enabled) return MODE_PLAIN;
     const bool two = s->pack.guards != s->pack.guards1;
-    if (forced == 0 && s->key.grouped) return two ? MODE_GROUPED2 : MODE_GROUPED;
+    if ((forced == 0 || forced == 4) && s->key.grouped) return two ? MODE_GROUPED2 : MODE_GROUPED;
     if (forced == 2 || !s->key.static_key) return two ? MODE_PACKED2 : MODE_PACKED;
     if (forced == 3 || !s->presorted) return two ? MODE_PACKED2_STATIC : MODE_PACKED_STATIC;
     return two ? MODE_SORTED2 : MODE_SORTED;
@@ -806,7 +966,9 @@ void fill_params(PlaceParams &p, const nbos_snapshot *s, const int32_t *d_reques
     p.feas = s->d_feas;
     p.ab = s->d_ab;
     p.pk = s->d_pk;
+    p.rk = s->d_rk;
     p.pack = s->pack;
+    p.rank = s->rank;
     p.requests = reinterpret_cast<const int4 *>(d_requests);
     p.out_hosts = d_out_hosts;
     p.out_found = d_out_found;
@@ -863,7 +1025,7 @@ int make_plan(const nbos_snapshot *s, long long total, long long batch, const nb
     int L = c.lanes_per_request;
     int blocks_per_sm = per_sm;
     {
-        const double pair_cost = mode_is_sorted(mode) ? 3.0 : mode_is_grouped(mode) ? 3.3 : mode_is_static(mode) ? 4.0 : mode_is_packed(mode) ? 5.0
+        const double pair_cost = (mode_is_sorted(mode) || mode_is_ranked(mode)) ? 3.0 : mode_is_grouped(mode) ? 3.3 : mode_is_static(mode) ? 4.0 : mode_is_packed(mode) ? 5.0
                                  : mode == MODE_PLAIN ? 7.0 : 12.0;
         const double kPassCost = 490.0, kRequestCost = 190.0, kHostCost = 1.6, kMergeCost = 12.0;
         const double issue_rate[4] = {0.376, 0.472, 0.499, 0.529};  // per scheduler, by resident blocks
@@ -940,8 +1102,8 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
         return fail(NBOS_ERR_INVALID_ARG, "requests_per_lane must be 1,2,4 or 8");
     if (c.host_split < 0 || c.grid_blocks < 0 || c.tile_hosts < 0 || (c.tile_hosts & 31))
         return fail(NBOS_ERR_INVALID_ARG, "launch config: negative field or tile_hosts not a multiple of 32");
-    if (c.pair_mode < 0 || c.pair_mode > 3)
-        return fail(NBOS_ERR_INVALID_ARG, "pair_mode must be 0 (automatic), 1 (plain compares), 2 (packed, key computed per pair) or 3 (packed, host key compared per pair)");
+    if (c.pair_mode < 0 || c.pair_mode > 4)
+        return fail(NBOS_ERR_INVALID_ARG, "pair_mode must be 0 (automatic), 1 (plain compares), 2 (packed, key computed per pair), 3 (packed, host key compared per pair) or 4 (key-order forms that retire requests)");
 
     if (c.first_fit && s->key.static_key && s->presorted) {
         FirstFitParams fp;

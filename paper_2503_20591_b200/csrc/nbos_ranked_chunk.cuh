@@ -1,0 +1,96 @@
+// Pair step of the placement kernel in its ranked form (see RankLayout in nbos_internal.h).
+//
+// A host and a request are one 64-bit value each: the four capacities of Section 3.2.1 and the
+// rank in the order of Section 3.4.1, every field under a guard bit. host - request leaves all
+// guards set exactly when the host fits the ask (coarsely, never rejecting a host that fits) and
+// ranks before the request's current third best. So a (request, host) pair costs one 64-bit
+// subtraction and one 3-input logic operation, ~(lo & hi) & guards, whose "result != 0"
+// predicate is chained through the pairs of a chunk: the chain stays true only while every pair
+// failed. Nothing else happens per pair; when some pair of a chunk passed, the caller re-tests
+// the chunk exactly and updates the best three.
+//
+// Pipe balance. The 64-bit subtraction is one integer-ALU instruction, and so is the logic
+// operation; the same subtraction done as two 32-bit multiply-adds with -1 (no borrow crosses
+// bit 31: a host word always has its top guard set, a request word never) runs on the multiply
+// pipe instead. Both pipes take a warp instruction every second cycle, so the requests of a
+// chunk are split between the two forms (NBOS_RANKED_FORMS, request by request: W = one 64-bit
+// subtraction, M = two multiply-adds).
+//
+// One asm statement covers a whole chunk (W hosts x Q requests) because a predicate cannot leave
+// an asm statement. Operands: %0 flag (out), %1..%8 requests, %9..%12 hosts, %13 guard mask.
+#ifndef NBOS_RANKED_CHUNK_CUH_
+#define NBOS_RANKED_CHUNK_CUH_
+
+namespace nbos {
+
+#define NBOS_RK_W(P, r, h)                                          \
+    "sub.u64 dd, %" #h ", %" #r ";\n\t"                             \
+    "mov.b64 {d0, d1}, dd;\n\t"                                     \
+    "lop3.and.b32 e|" #P ", d0, d1, %13, 0x2a, " #P ";\n\t"
+#define NBOS_RK_M(P, r, h)                                          \
+    "mov.b64 {r0, r1}, %" #r ";\n\t"                                \
+    "mov.b64 {h0, h1}, %" #h ";\n\t"                                \
+    "mad.lo.u32 d0, r0, 0xffffffff, h0;\n\t"                        \
+    "mad.lo.u32 d1, r1, 0xffffffff, h1;\n\t"                        \
+    "lop3.and.b32 e|" #P ", d0, d1, %13, 0x2a, " #P ";\n\t"
+
+// form of request 1..8 of a row (chosen by timing)
+#ifndef NBOS_RANKED_FORMS
+#define NBOS_RK_F1 NBOS_RK_M
+#define NBOS_RK_F2 NBOS_RK_W
+#define NBOS_RK_F3 NBOS_RK_M
+#define NBOS_RK_F4 NBOS_RK_M
+#define NBOS_RK_F5 NBOS_RK_W
+#define NBOS_RK_F6 NBOS_RK_M
+#define NBOS_RK_F7 NBOS_RK_M
+#define NBOS_RK_F8 NBOS_RK_W
+#endif
+
+// rows: one host against the first Q requests; four predicate chains take turns
+#define NBOS_RK_ROW1(h) NBOS_RK_F1(p0, 1, h)
+#define NBOS_RK_ROW2(h) NBOS_RK_ROW1(h) NBOS_RK_F2(p1, 2, h)
+#define NBOS_RK_ROW4(h) NBOS_RK_ROW2(h) NBOS_RK_F3(p2, 3, h) NBOS_RK_F4(p3, 4, h)
+#define NBOS_RK_ROW8(h) \
+    NBOS_RK_ROW4(h) NBOS_RK_F5(p0, 5, h) NBOS_RK_F6(p1, 6, h) NBOS_RK_F7(p2, 7, h) NBOS_RK_F8(p3, 8, h)
+#define NBOS_RK_HOSTS1(ROW) ROW(9)
+#define NBOS_RK_HOSTS4(ROW) ROW(9) ROW(10) ROW(11) ROW(12)
+
+#define NBOS_RK_CHUNK_ASM(BODY)                                                                      \
+    asm volatile(                                                                                    \
+        "{\n\t.reg .pred p0, p1, p2, p3;\n\t.reg .u32 d0, d1, r0, r1, h0, h1, e;\n\t.reg .b64 dd;\n\t" \
+        "setp.eq.u32 p0, 0, 0;\n\tsetp.eq.u32 p1, 0, 0;\n\t"                                         \
+        "setp.eq.u32 p2, 0, 0;\n\tsetp.eq.u32 p3, 0, 0;\n\t" BODY                                    \
+        "and.pred p0, p0, p1;\n\tand.pred p2, p2, p3;\n\tand.pred p0, p0, p2;\n\t"                  \
+        "selp.u32 %0, 0, 1, p0;\n\t}"                                                                \
+        : "=r"(any_pass)                                                                             \
+        : "l"(a[0]), "l"(a[1]), "l"(a[2]), "l"(a[3]), "l"(a[4]), "l"(a[5]), "l"(a[6]), "l"(a[7]),    \
+          "l"(x[0]), "l"(x[1]), "l"(x[2]), "l"(x[3]), "r"(guards))
+
+// True when at least one of the W x Q (host, request) pairs of the chunk keeps all its guards.
+template <int Q, int W>
+__device__ __forceinline__ bool ranked_chunk_any_pass(const unsigned long long (&rq)[Q],
+                                                      const unsigned long long (&h)[W], unsigned int guards)
+{
+    static_assert((Q == 1 || Q == 2 || Q == 4 || Q == 8) && (W == 1 || W == 4), "chunk shape");
+    unsigned long long a[8], x[4];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) a[q] = q < Q ? rq[q] : 0ull;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) x[u] = u < W ? h[u] : 0ull;
+    unsigned int any_pass;
+#define NBOS_RK_CASE(QV, ROW)                                                   \
+    if constexpr (Q == QV) {                                                    \
+        if constexpr (W == 4) NBOS_RK_CHUNK_ASM(NBOS_RK_HOSTS4(ROW));           \
+        else NBOS_RK_CHUNK_ASM(NBOS_RK_HOSTS1(ROW));                            \
+    }
+    NBOS_RK_CASE(1, NBOS_RK_ROW1)
+    NBOS_RK_CASE(2, NBOS_RK_ROW2)
+    NBOS_RK_CASE(4, NBOS_RK_ROW4)
+    NBOS_RK_CASE(8, NBOS_RK_ROW8)
+#undef NBOS_RK_CASE
+    return any_pass != 0u;
+}
+
+}  // namespace nbos
+
+#endif  // NBOS_RANKED_CHUNK_CUH_
