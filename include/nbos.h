@@ -122,6 +122,12 @@ typedef struct nbos_snapshot_info {
     int32_t grouped;     /* 1: hosts differ in GPU count; the table is stored count by count,
                           * each group in ascending key order                               */
     int64_t workspace_bytes;
+    int32_t ranked;      /* 1: the ranked form is available (static_key and presorted): capacities and
+                          * the host's rank in the order of Section 3.4.1 packed into one 64-bit
+                          * value per host, compared with one subtraction per pair               */
+    int32_t ranked_dropped_bits[4]; /* low bits of (GPUs, VRAM, millicpus, memory) the ranked form
+                          * leaves out of its per-pair test; pairs that pass are re-tested exactly */
+    int32_t reserved;
 } nbos_snapshot_info;
 
 /*

@@ -70,6 +70,8 @@ class nbos_snapshot_info(ctypes.Structure):
         ("packed_test", ctypes.c_int32), ("static_key", ctypes.c_int32),
         ("presorted", ctypes.c_int32), ("grouped", ctypes.c_int32),
         ("workspace_bytes", ctypes.c_int64),
+        ("ranked", ctypes.c_int32), ("ranked_dropped_bits", ctypes.c_int32 * 4),
+        ("reserved", ctypes.c_int32),
     ]
 
 

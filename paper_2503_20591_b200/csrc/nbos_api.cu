@@ -340,6 +340,9 @@ int nbos_snapshot_get_info(const nbos_snapshot *s, nbos_snapshot_info *out)
     out->presorted = s->presorted;
     out->grouped = s->key.grouped;
     out->workspace_bytes = (int64_t)s->workspace_bytes;
+    out->ranked = s->rank.enabled;
+    for (int c = 0; c < 4; ++c) out->ranked_dropped_bits[c] = s->rank.enabled ? s->rank.fdrop[c] : 0;
+    out->reserved = 0;
     return NBOS_OK;
 }
 

@@ -517,7 +517,8 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
     };
 
     unsigned long long rq[Q];
-    unsigned int t1[Q], t2[Q], t3[Q];
+    unsigned int best[3 * Q];  // positions of the best three: [0, Q) best, [Q, 2Q) second, [2Q, 3Q) third
+    unsigned int field[Q];     // rank field of each request after an update
 #pragma unroll
     for (int q = 0; q < Q; ++q) {
         const int4 r = load_request(q);
@@ -535,7 +536,8 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
             if (p.rank.fword[k]) w1 |= piece; else w0 |= piece;
         }
         rq[q] = (unsigned long long)w0 | ((unsigned long long)w1 << 32);  // rank field 0: every rank passes
-        t1[q] = kNone; t2[q] = kNone; t3[q] = kNone;
+        best[q] = kNone; best[Q + q] = kNone; best[2 * Q + q] = kNone;
+        field[q] = 0u;
     }
 
     const int T = p.tile_hosts;
@@ -560,21 +562,28 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
                 for (int u = 0; u < W; ++u) h[u] = R[i0 + u * L];
             }
             if (ranked_chunk_any_pass<Q, W>(rq, h, guards)) {
-                // rare: exact re-test of the chunk's pairs, then the new thresholds
+                // rare: exact re-test of the chunk's pairs, then the new thresholds. The loop over
+                // the requests is deliberately not unrolled: the best-three arrays are then indexed
+                // dynamically and live in local memory, which keeps their 3 * Q registers out of
+                // the pair loop.
                 int4 f[W];
 #pragma unroll
                 for (int u = 0; u < W; ++u) f[u] = __ldg(p.feas + row + pos0 + i0 + u * L);
-#pragma unroll
+#pragma unroll 1
                 for (int q = 0; q < Q; ++q) {
                     const int4 r = load_request(q);
+                    unsigned int a1 = best[q], a2 = best[Q + q], a3 = best[2 * Q + q];
 #pragma unroll
                     for (int u = 0; u < W; ++u) {
                         const bool ok = (r.x <= f[u].x) & (r.y <= f[u].y) & (r.z <= f[u].z) & (r.w <= f[u].w);
-                        insert3(t1[q], t2[q], t3[q], ok ? (unsigned int)(pos0 + i0 + u * L) : kNone);
+                        insert3(a1, a2, a3, ok ? (unsigned int)(pos0 + i0 + u * L) : kNone);
                     }
-                    const unsigned int field = t3[q] == kNone ? 0u : p.rank.rank_top + 1u - t3[q];
-                    rq[q] = (rq[q] & ~rank_mask) | ((unsigned long long)field << rank_shift);
+                    best[q] = a1; best[Q + q] = a2; best[2 * Q + q] = a3;
+                    field[q] = a3 == kNone ? 0u : p.rank.rank_top + 1u - a3;
                 }
+#pragma unroll
+                for (int q = 0; q < Q; ++q)
+                    rq[q] = (rq[q] & ~rank_mask) | ((unsigned long long)field[q] << rank_shift);
             }
         };
         int i = sub;
@@ -585,6 +594,9 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
     }
 
     // merge the L lanes of a group (positions are unique)
+    unsigned int t1[Q], t2[Q], t3[Q];
+#pragma unroll
+    for (int q = 0; q < Q; ++q) { t1[q] = best[q]; t2[q] = best[Q + q]; t3[q] = best[2 * Q + q]; }
 #pragma unroll
     for (int mask = 1; mask < L; mask <<= 1) {
 #pragma unroll

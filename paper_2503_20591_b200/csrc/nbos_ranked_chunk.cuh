@@ -34,16 +34,50 @@ namespace nbos {
     "mad.lo.u32 d1, r1, 0xffffffff, h1;\n\t"                        \
     "lop3.and.b32 e|" #P ", d0, d1, %13, 0x2a, " #P ";\n\t"
 
-// form of request 1..8 of a row (chosen by timing)
-#ifndef NBOS_RANKED_FORMS
+// form of request 1..8 of a row: bit q-1 of NBOS_RK_PATTERN set = request q takes the 64-bit
+// subtraction (chosen by timing)
+#ifndef NBOS_RK_PATTERN
+#define NBOS_RK_PATTERN 0x92
+#endif
+#if NBOS_RK_PATTERN & 0x01
+#define NBOS_RK_F1 NBOS_RK_W
+#else
 #define NBOS_RK_F1 NBOS_RK_M
+#endif
+#if NBOS_RK_PATTERN & 0x02
 #define NBOS_RK_F2 NBOS_RK_W
+#else
+#define NBOS_RK_F2 NBOS_RK_M
+#endif
+#if NBOS_RK_PATTERN & 0x04
+#define NBOS_RK_F3 NBOS_RK_W
+#else
 #define NBOS_RK_F3 NBOS_RK_M
+#endif
+#if NBOS_RK_PATTERN & 0x08
+#define NBOS_RK_F4 NBOS_RK_W
+#else
 #define NBOS_RK_F4 NBOS_RK_M
+#endif
+#if NBOS_RK_PATTERN & 0x10
 #define NBOS_RK_F5 NBOS_RK_W
+#else
+#define NBOS_RK_F5 NBOS_RK_M
+#endif
+#if NBOS_RK_PATTERN & 0x20
+#define NBOS_RK_F6 NBOS_RK_W
+#else
 #define NBOS_RK_F6 NBOS_RK_M
+#endif
+#if NBOS_RK_PATTERN & 0x40
+#define NBOS_RK_F7 NBOS_RK_W
+#else
 #define NBOS_RK_F7 NBOS_RK_M
+#endif
+#if NBOS_RK_PATTERN & 0x80
 #define NBOS_RK_F8 NBOS_RK_W
+#else
+#define NBOS_RK_F8 NBOS_RK_M
 #endif
 
 // rows: one host against the first Q requests; four predicate chains take turns

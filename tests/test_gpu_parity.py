@@ -129,10 +129,12 @@ def test_key_widths_orders_flags(nb, lib_flags, key_order, flags):
             assert_same(got, ref, f"{w.name} order={key_order} flags={flags} lib={lib_flags}")
 
 
-@pytest.mark.parametrize("pair_mode", [0, 1, 2, 3])
+@pytest.mark.parametrize("pair_mode", [0, 1, 2, 3, 4])
 @pytest.mark.parametrize("lanes", [0, 1, 4, 32])
 def test_pair_evaluation_modes(nb, pair_mode, lanes):
-    """Plain compares, packed test with per-pair key, and the automatic choice give the same bytes."""
+    """Plain compares, packed test with the key computed or compared per pair, the key-order forms
+    that retire requests, and the automatic choice (ranked form where available) give the same
+    bytes."""
     cfg = nb.launch_config(lanes_per_request=lanes, pair_mode=pair_mode)
     for w in (W.make_config(2, batch=6000), W.mixed_gpu_cluster(900, 2500, seed=31),
               W.make_config(4, batch=80, n_snapshots=40), W.make_config(3, batch=3000)):
@@ -183,6 +185,59 @@ def test_packed_test_layouts_and_fallback(nb):
         w5.requests[0, 2 * k + 1, k] = top + 1
     got, ref = both(nb, w5)
     assert_same(got, ref, "asks at the capacity maxima")
+
+
+def test_ranked_form_coarse_fields(nb):
+    """Ranked form: capacities wider than their field lose low bits in the per-pair test, and a
+    pair that passes it is re-tested exactly. Workloads built so that asks and capacities often
+    fall into the same coarse bucket (the coarse test passes, the exact one may not), in every
+    resource, with every launch shape; same bytes as the checker."""
+    rng = np.random.default_rng(77)
+    shapes = (dict(), dict(lanes_per_request=1), dict(lanes_per_request=4, requests_per_lane=2),
+              dict(lanes_per_request=32, tile_hosts=64), dict(lanes_per_request=2, host_split=3, tile_hosts=64))
+    # (a) cfg3-like cluster: millicpus / memory capacities and asks crowd around the same values
+    w = W.make_config(3, batch=4000)
+    h = w.n_hosts
+    w.millicpus[0, :] = 100_000 + rng.integers(0, 64, size=h)
+    w.mem_mb[0, :] = 1_000_000 + rng.integers(0, 4096, size=h)
+    w.requests[0, :, 2] = 100_000 + rng.integers(0, 64, size=w.batch)
+    w.requests[0, :, 3] = 1_000_000 + rng.integers(0, 4096, size=w.batch)
+    w.requests[0, :64, 3] = 1_000_000 + 4094      # only a handful of hosts have that much
+    s = nb.snapshot_from_workload(w)
+    info = s.info()
+    nb.nbos_snapshot_destroy(s)
+    assert info.ranked == 1 and info.static_key == 1 and info.presorted == 1
+    assert info.ranked_dropped_bits[0] == 0          # the GPU component is always exact
+    assert max(info.ranked_dropped_bits[1:]) > 0     # something is coarse at this size
+    for shape in shapes:
+        got, ref = both(nb, w, config=nb.launch_config(**shape) if shape else None)
+        assert_same(got, ref, f"crowded capacities {shape}")
+    assert (ref[1] == 3).any() and (ref[1] < 3).any()
+    # (b) capacities near 2^31: most bits dropped
+    w2 = W.make_config(1, batch=3000)
+    w2.mem_mb[0, :] = (1 << 31) - 1 - rng.integers(0, 1 << 16, size=w2.n_hosts)
+    w2.millicpus[0, :] = (1 << 30) + rng.integers(0, 1 << 12, size=w2.n_hosts)
+    w2.requests[0, :, 3] = (1 << 31) - 1 - rng.integers(0, 1 << 16, size=w2.batch)
+    w2.requests[0, :, 2] = (1 << 30) + rng.integers(0, 1 << 12, size=w2.batch)
+    s = nb.snapshot_from_workload(w2)
+    info = s.info()
+    nb.nbos_snapshot_destroy(s)
+    assert info.ranked == 1 and info.packed_test == 0 and min(info.ranked_dropped_bits[2:]) >= 8
+    for shape in shapes:
+        for key_order in (0, 1):
+            got, ref = both(nb, w2, key_order=key_order, config=nb.launch_config(**shape) if shape else None)
+            assert_same(got, ref, f"wide capacities {shape} order={key_order}")
+    # (c) VRAM crowded too, idle reading, several snapshots with different limits
+    w3 = W.make_config(4, batch=300, n_snapshots=12)
+    w3.vram_gb[:, :] = 600 + rng.integers(0, 40, size=w3.vram_gb.shape)
+    w3.requests[:, :, 1] = 600 + rng.integers(0, 40, size=w3.requests.shape[:2])
+    for flags in (0, 1):
+        got, ref = both(nb, w3, flags=flags)
+        assert_same(got, ref, f"crowded VRAM flags={flags}")
+    # (d) mixed GPU counts have no ranked form (hosts rank differently for different asks)
+    s = nb.snapshot_from_workload(W.mixed_gpu_cluster(300, 100, seed=8))
+    assert s.info().ranked == 0
+    nb.nbos_snapshot_destroy(s)
 
 
 def test_tables_grouped_by_gpu_count(nb):
