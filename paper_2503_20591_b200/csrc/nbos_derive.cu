@@ -302,6 +302,7 @@ struct FinalizeArgs {
     void *ab;
     uint4 *pk;
     uint2 *rk;
+    unsigned int *rk1;
     int Hpad;
     PackLayout pack;
     RankLayout ranked;
@@ -336,6 +337,13 @@ __global__ void __launch_bounds__(256) finalize_kernel(const FinalizeArgs a)
         for (int c = 0; c < 4; ++c) w[a.ranked.fword[c]] |= (cap[c] >> a.ranked.fdrop[c]) << a.ranked.fshift[c];
         w[a.ranked.fword[4]] |= (a.ranked.rank_top - j) << a.ranked.fshift[4];
         a.rk[base + j] = make_uint2(w[0], w[1]);
+        if (a.ranked.l1_enabled) {
+            unsigned int w1 = a.ranked.l1_guards;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) w1 |= (cap[c] >> a.ranked.l1_drop[c]) << a.ranked.l1_shift[c];
+            w1 |= (a.ranked.rank_top - j) << a.ranked.l1_shift[4];
+            a.rk1[base + j] = w1;
+        }
     }
 }
 
@@ -376,6 +384,7 @@ Layout workspace_layout(int N, int Hpad)
     l.off_ab = o;      o = up(o + (size_t)N * Hpad * sizeof(ulonglong2));
     l.off_pk = o;      o = up(o + (size_t)N * Hpad * sizeof(uint4));
     l.off_rk = o;      o = up(o + (size_t)N * Hpad * sizeof(uint2));
+    l.off_rk1 = o;     o = up(o + (size_t)N * Hpad * sizeof(unsigned int));
     l.off_tmp_feas = o; o = up(o + (size_t)N * Hpad * sizeof(int4));
     l.off_tmp_ab = o;  o = up(o + (size_t)N * Hpad * sizeof(ulonglong2));
     l.off_tmp_seq = o; o = up(o + (size_t)N * Hpad * sizeof(int4));
@@ -470,7 +479,8 @@ int emit_tables(DeriveCtx &c)
         rank_kernel<<<dim3((Hpad + 255) / 256, (Hpad + kRankChunk - 1) / kRankChunk, N), 256, 0, c.stream>>>(sortkey, perm, Hpad);
     FinalizeArgs fa{tmp_feas, tmp_ab, s->presorted ? perm : nullptr, reinterpret_cast<int4 *>(c.ws + c.lay.off_feas),
                     c.ws + c.lay.off_ab, reinterpret_cast<uint4 *>(c.ws + c.lay.off_pk),
-                    reinterpret_cast<uint2 *>(c.ws + c.lay.off_rk), Hpad, s->pack, s->rank};
+                    reinterpret_cast<uint2 *>(c.ws + c.lay.off_rk),
+                    reinterpret_cast<unsigned int *>(c.ws + c.lay.off_rk1), Hpad, s->pack, s->rank};
     if (k.key_bits == 32)
         finalize_kernel<uint2><<<grid, 256, 0, c.stream>>>(fa);
     else
@@ -666,6 +676,37 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
             for (int c2 = 0; c2 < 4; ++c2) rl.fmax[c2] = field_max[c2];
             rl.rank_top = (unsigned int)(Hpad - 1);
             rl.rank_mask = ((1u << w6[4]) - 1u) << rl.fshift[4];
+            // first level: five fields + five guards in 32 bits. The GPU component and the rank
+            // keep their widths; the three other capacities share what is left as evenly as
+            // their widths allow (a component narrower than its share passes the rest on).
+            int left = 32 - 5 - w6[0] - w6[4];
+            if (left >= 3) {
+                int give[4] = {w6[0], 0, 0, 0};
+                int need[4] = {0, w6[1], w6[2], w6[3]};
+                while (left > 0) {
+                    int pick = -1;  // the component that still lacks the most bits
+                    for (int c2 = 1; c2 < 4; ++c2)
+                        if (need[c2] > give[c2] && (pick < 0 || give[c2] < give[pick] ||
+                                                    (give[c2] == give[pick] && need[c2] > need[pick])))
+                            pick = c2;
+                    if (pick < 0) break;
+                    ++give[pick];
+                    --left;
+                }
+                int at = 0;
+                rl.l1_enabled = 1;
+                rl.l1_guards = 0u;
+                for (int c2 = 1; c2 <= 5; ++c2) {      // order: VRAM, millicpus, memory, GPUs, rank
+                    const int comp = c2 <= 3 ? c2 : c2 == 4 ? 0 : 4;
+                    const int wdt = comp == 4 ? w6[4] : give[comp];
+                    rl.l1_shift[comp] = at;
+                    rl.l1_drop[comp] = comp == 4 ? 0 : w6[comp] - wdt;
+                    at += wdt;
+                    rl.l1_guards |= 1u << at;
+                    ++at;
+                }
+                rl.l1_rank_mask = ((1u << w6[4]) - 1u) << rl.l1_shift[4];
+            }
         }
     }
     s->rank = rl;
@@ -688,6 +729,7 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     s->d_ab = c.ws + c.lay.off_ab;
     s->d_pk = reinterpret_cast<const uint4 *>(c.ws + c.lay.off_pk);
     s->d_rk = reinterpret_cast<const uint2 *>(c.ws + c.lay.off_rk);
+    s->d_rk1 = reinterpret_cast<const unsigned int *>(c.ws + c.lay.off_rk1);
     s->d_host_feas = reinterpret_cast<const int4 *>(c.ws + c.lay.off_tmp_feas);
     s->d_host_ab = c.ws + c.lay.off_tmp_ab;
     s->d_host_seq = reinterpret_cast<const int4 *>(c.ws + c.lay.off_tmp_seq);

@@ -42,7 +42,7 @@ enum : unsigned int {
 };
 
 struct Layout {
-    size_t off_status, off_limits, off_sums, off_stats, off_lambda, off_g_single, off_feas, off_ab, off_pk, off_rk;
+    size_t off_status, off_limits, off_sums, off_stats, off_lambda, off_g_single, off_feas, off_ab, off_pk, off_rk, off_rk1;
     size_t off_tmp_feas, off_tmp_ab, off_tmp_seq, off_sortkey, off_perm, total;
 };
 Layout workspace_layout(int n_snapshots, int hosts_padded);
@@ -92,6 +92,14 @@ struct RankLayout {
     unsigned int guards;    // guard bits, the same in both words
     unsigned int rank_top;  // host field = rank_top - position in the table
     unsigned int rank_mask; // bits of the rank field inside its word
+    // First level: the same five fields once more in a single 32-bit word per host (each under its
+    // own guard bit; the GPU component and the rank exact, the three other capacities with as many
+    // of their high bits as are left). One 32-bit subtraction and one logic operation per pair
+    // answer "cannot enter the best three" for most pairs; only chunks in which some pair
+    // passes go on to the two-word test above.
+    int l1_enabled;
+    int l1_shift[5], l1_drop[5];
+    unsigned int l1_guards, l1_rank_mask;
 };
 
 }  // namespace nbos
@@ -109,6 +117,7 @@ struct nbos_snapshot {
     const uint4 *d_pk;    // [N][Hpad] (word0, word1, A, B), only when pack.enabled
     nbos::PackLayout pack;
     const uint2 *d_rk;    // [N][Hpad] (word0, word1) of the ranked form, only when rank.enabled
+    const unsigned int *d_rk1;  // [N][Hpad] first-level word of the ranked form, only when rank.l1_enabled
     nbos::RankLayout rank;
     int presorted;
     int idle_max;             // the key's idle field stores idle_max - (G - C)

@@ -57,9 +57,12 @@ enum : int {
     MODE_RANKED = 10,        // static key, table in key order: capacities and rank in one 64-bit value per
                              // host and per request, one subtraction + one logic operation per pair;
                              // pairs that pass are re-tested exactly          (records: rk, then feas + ab)
-    MODE_COUNT = 11,
+    MODE_RANKED2 = 11,       // as 10 behind a first level: one 32-bit word per host and per request, one
+                             // subtraction + one logic operation per pair; chunks in which a pair passes
+                             // go through the two-word test               (records: rk + rk1, then feas + ab)
+    MODE_COUNT = 12,
 };
-__host__ __device__ constexpr bool mode_is_ranked(int mode) { return mode == MODE_RANKED; }
+__host__ __device__ constexpr bool mode_is_ranked(int mode) { return mode == MODE_RANKED || mode == MODE_RANKED2; }
 __host__ __device__ constexpr bool mode_is_packed(int mode) { return mode >= MODE_PACKED && mode <= MODE_GROUPED2; }
 __host__ __device__ constexpr bool mode_is_sorted(int mode) { return mode == MODE_SORTED || mode == MODE_SORTED2; }
 __host__ __device__ constexpr bool mode_is_grouped(int mode) { return mode == MODE_GROUPED || mode == MODE_GROUPED2; }
@@ -67,7 +70,7 @@ __host__ __device__ constexpr bool mode_is_grouped(int mode) { return mode == MO
 __host__ __device__ constexpr bool mode_is_chained(int mode) { return mode_is_sorted(mode) || mode_is_grouped(mode); }
 __host__ __device__ constexpr bool mode_is_static(int mode) { return mode == MODE_PACKED_STATIC || mode == MODE_PACKED2_STATIC || mode_is_sorted(mode); }
 __host__ __device__ constexpr bool mode_two_masks(int mode) { return mode == MODE_PACKED2 || mode == MODE_PACKED2_STATIC || mode == MODE_SORTED2 || mode == MODE_GROUPED2; }
-__host__ __device__ constexpr int mode_record_bytes(int mode) { return mode == MODE_KEY64 ? 32 : mode == MODE_PLAIN ? 24 : mode == MODE_RANKED ? 8 : 16; }
+__host__ __device__ constexpr int mode_record_bytes(int mode) { return mode == MODE_KEY64 ? 32 : mode == MODE_PLAIN ? 24 : mode == MODE_RANKED ? 8 : mode == MODE_RANKED2 ? 12 : 16; }
 __host__ __device__ constexpr int mode_max_q(int mode) { return mode == MODE_KEY64 ? 4 : 8; }
 // Resident blocks per SM the kernels are compiled for. The modes that rank hosts by their own key
 // touch most best-three registers only on the rare update path, so 64 registers (a few spills
@@ -80,7 +83,8 @@ struct PlaceParams {
     const int4 *feas;       // [N][Hpad]
     const void *ab;         // [N][Hpad] pairs (A, B)
     const uint4 *pk;        // [N][Hpad] (word0, word1, A, B), packed modes
-    const uint2 *rk;        // [N][Hpad] (word0, word1), ranked mode
+    const uint2 *rk;        // [N][Hpad] (word0, word1), ranked modes
+    const unsigned int *rk1;  // [N][Hpad] first-level word, MODE_RANKED2
     PackLayout pack;
     RankLayout rank;
     const int4 *requests;   // [N * B]
@@ -485,11 +489,12 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
 // ---- one pass in ranked form ------------------------------------------------------------------
 // Same contract as run_pass. The best three of a request are kept as positions in the table
 // (which is stored in key order, so a smaller position is a smaller key) and turned into keys
-// after the last tile. Per pair: ranked_chunk_any_pass. When a chunk reports a pass, its pairs
-// are re-tested with the exact records (four compares against the request as it was given),
-// fitting hosts enter the best three, and the request's rank field is set from its new third
-// best.
-template <int Q, int L>
+// after the last tile. Per pair: one subtraction and one logic operation on the first-level
+// words (TWO_LEVELS), or directly the two-word test. A chunk in which some pair passed the first
+// level goes through the two-word test; pairs that pass that one too are re-tested with the exact
+// records (four compares against the request as it was given), fitting hosts enter the best
+// three, and the request's rank fields are set from its new third best.
+template <int Q, int L, bool TWO_LEVELS>
 __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned char *stages,
                                                 uint32_t stage_bytes, uint32_t full_bar,
                                                 uint32_t empty_bar, volatile unsigned int *abort_flag,
@@ -504,6 +509,7 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
     const int lane = tid & 31;
     const size_t row = (size_t)n * p.Hpad;
     const unsigned int guards = p.rank.guards;
+    const unsigned int guards1 = p.rank.l1_guards;
     const int rank_shift = p.rank.fshift[4] + 32 * p.rank.fword[4];
     const unsigned long long rank_mask = (unsigned long long)p.rank.rank_mask << (32 * p.rank.fword[4]);
 
@@ -516,7 +522,8 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
         return r;
     };
 
-    unsigned long long rq[Q];
+    unsigned long long rq[Q];              // two-word form of each request
+    unsigned int r1[TWO_LEVELS ? Q : 1];   // first-level word
     unsigned int best[3 * Q];  // positions of the best three: [0, Q) best, [Q, 2Q) second, [2Q, 3Q) third
     unsigned int field[Q];     // rank field of each request after an update
 #pragma unroll
@@ -529,13 +536,15 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
         const unsigned int val[4] = {bad ? (unsigned int)p.rank.fmax[0] + 2u : (unsigned int)r.x + 1u,
                                      bad ? 0u : (unsigned int)r.y, bad ? 0u : (unsigned int)r.z,
                                      bad ? 0u : (unsigned int)r.w};
-        unsigned int w0 = 0u, w1 = 0u;
+        unsigned int w0 = 0u, w1 = 0u, l1 = 0u;
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             const unsigned int piece = (val[k] >> p.rank.fdrop[k]) << p.rank.fshift[k];
             if (p.rank.fword[k]) w1 |= piece; else w0 |= piece;
+            l1 |= (val[k] >> p.rank.l1_drop[k]) << p.rank.l1_shift[k];
         }
         rq[q] = (unsigned long long)w0 | ((unsigned long long)w1 << 32);  // rank field 0: every rank passes
+        if constexpr (TWO_LEVELS) r1[q] = l1;
         best[q] = kNone; best[Q + q] = kNone; best[2 * Q + q] = kNone;
         field[q] = 0u;
     }
@@ -546,10 +555,13 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
         const uint32_t parity = (ring_pos / kStages) & 1u;
         if (!mbar_wait(full_bar + 8u * s, parity, abort_flag)) return false;
         const unsigned long long *R = reinterpret_cast<const unsigned long long *>(stages + (size_t)s * stage_bytes);
+        const unsigned int *R1 = reinterpret_cast<const unsigned int *>(R + T);
         const int pos0 = t * T;
         int hosts = p.Hpad - pos0;
         if (hosts > T) hosts = T;
-        auto chunk = [&](auto width, int i0) {
+
+        // two-word test of W hosts (i0, i0 + L, ...) against the Q requests, then the exact part
+        auto chunk2 = [&](auto width, int i0) {
             constexpr int W = decltype(width)::value;
             unsigned long long h[W];
             if constexpr (L == 1 && W == 4) {
@@ -561,34 +573,75 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
 #pragma unroll
                 for (int u = 0; u < W; ++u) h[u] = R[i0 + u * L];
             }
-            if (ranked_chunk_any_pass<Q, W>(rq, h, guards)) {
-                // rare: exact re-test of the chunk's pairs, then the new thresholds. The loop over
-                // the requests is deliberately not unrolled: the best-three arrays are then indexed
-                // dynamically and live in local memory, which keeps their 3 * Q registers out of
-                // the pair loop.
-                int4 f[W];
+            if (!ranked_chunk_any_pass<Q, W>(rq, h, guards)) return;
+            // rare. Which pairs passed (bit q * W + u), with static register indices ...
+            unsigned int passed = 0u;
 #pragma unroll
-                for (int u = 0; u < W; ++u) f[u] = __ldg(p.feas + row + pos0 + i0 + u * L);
-#pragma unroll 1
-                for (int q = 0; q < Q; ++q) {
-                    const int4 r = load_request(q);
+            for (int q = 0; q < Q; ++q)
+#pragma unroll
+                for (int u = 0; u < W; ++u) {
+                    const unsigned long long d = h[u] - rq[q];
+                    const unsigned int fell = ~((unsigned int)d & (unsigned int)(d >> 32)) & guards;
+                    passed |= (fell == 0u ? 1u : 0u) << (q * W + u);
+                }
+            // ... then one pair after the other: exact test against the request as given; the
+            // best-three arrays are indexed dynamically here and therefore live in local memory,
+            // which keeps their 3 * Q registers out of the pair loop
+            unsigned int touched = 0u;
+            while (passed) {
+                const int bit = __ffs(passed) - 1;
+                passed &= passed - 1u;
+                const int q = bit / W, u = bit % W;
+                const unsigned int pos = (unsigned int)(pos0 + i0 + u * L);
+                const int4 r = load_request(q);
+                const int4 f = __ldg(p.feas + row + pos);
+                if ((r.x <= f.x) & (r.y <= f.y) & (r.z <= f.z) & (r.w <= f.w)) {
                     unsigned int a1 = best[q], a2 = best[Q + q], a3 = best[2 * Q + q];
-#pragma unroll
-                    for (int u = 0; u < W; ++u) {
-                        const bool ok = (r.x <= f[u].x) & (r.y <= f[u].y) & (r.z <= f[u].z) & (r.w <= f[u].w);
-                        insert3(a1, a2, a3, ok ? (unsigned int)(pos0 + i0 + u * L) : kNone);
-                    }
+                    insert3(a1, a2, a3, pos);
                     best[q] = a1; best[Q + q] = a2; best[2 * Q + q] = a3;
                     field[q] = a3 == kNone ? 0u : p.rank.rank_top + 1u - a3;
+                    touched = 1u;
                 }
+            }
+            if (touched) {
 #pragma unroll
-                for (int q = 0; q < Q; ++q)
+                for (int q = 0; q < Q; ++q) {
                     rq[q] = (rq[q] & ~rank_mask) | ((unsigned long long)field[q] << rank_shift);
+                    if constexpr (TWO_LEVELS) r1[q] = (r1[q] & ~p.rank.l1_rank_mask) | (field[q] << p.rank.l1_shift[4]);
+                }
             }
         };
+
         int i = sub;
-        for (; i + 3 * L < hosts; i += 4 * L) chunk(std::integral_constant<int, 4>{}, i);
-        for (; i < hosts; i += L) chunk(std::integral_constant<int, 1>{}, i);
+        if constexpr (TWO_LEVELS) {
+            auto chunk1 = [&](auto width, int i0) {
+                constexpr int W = decltype(width)::value;
+                unsigned int h1[W];
+                if constexpr (L == 1 && W == 8) {
+                    const uint4 a = *reinterpret_cast<const uint4 *>(R1 + i0);
+                    const uint4 b = *reinterpret_cast<const uint4 *>(R1 + i0 + 4);
+                    h1[0] = a.x; h1[1] = a.y; h1[2] = a.z; h1[3] = a.w;
+                    h1[4] = b.x; h1[5] = b.y; h1[6] = b.z; h1[7] = b.w;
+                } else {
+#pragma unroll
+                    for (int u = 0; u < W; ++u) h1[u] = R1[i0 + u * L];
+                }
+                if (ranked_l1_chunk_any_pass<Q, W>(r1, h1, guards1)) {
+                    if constexpr (W == 8) {
+                        chunk2(std::integral_constant<int, 4>{}, i0);
+                        chunk2(std::integral_constant<int, 4>{}, i0 + 4 * L);
+                    } else {
+                        chunk2(std::integral_constant<int, W>{}, i0);
+                    }
+                }
+            };
+            for (; i + 7 * L < hosts; i += 8 * L) chunk1(std::integral_constant<int, 8>{}, i);
+            for (; i + 3 * L < hosts; i += 4 * L) chunk1(std::integral_constant<int, 4>{}, i);
+            for (; i < hosts; i += L) chunk1(std::integral_constant<int, 1>{}, i);
+        } else {
+            for (; i + 3 * L < hosts; i += 4 * L) chunk2(std::integral_constant<int, 4>{}, i);
+            for (; i < hosts; i += L) chunk2(std::integral_constant<int, 1>{}, i);
+        }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty_bar + 8u * s);
     }
@@ -698,8 +751,11 @@ place_kernel(const __grid_constant__ PlaceParams p)
                 const uint32_t dst = stage0 + s * stage_bytes;
                 if (mode_is_ranked(MODE)) {
                     const uint32_t bytes = (uint32_t)hosts * 8u;
-                    mbar_arrive_expect_tx(full_bar + 8u * s, bytes);
+                    const uint32_t bytes1 = MODE == MODE_RANKED2 ? (uint32_t)hosts * 4u : 0u;
+                    mbar_arrive_expect_tx(full_bar + 8u * s, bytes + bytes1);
                     bulk_copy_g2s(dst, p.rk + row + (size_t)t * T, bytes, full_bar + 8u * s);
+                    if (MODE == MODE_RANKED2)
+                        bulk_copy_g2s(dst + (uint32_t)T * 8u, p.rk1 + row + (size_t)t * T, bytes1, full_bar + 8u * s);
                 } else if (kPacked) {
                     const uint32_t bytes = (uint32_t)hosts * 16u;
                     mbar_arrive_expect_tx(full_bar + 8u * s, bytes);
@@ -737,7 +793,7 @@ place_kernel(const __grid_constant__ PlaceParams p)
     while (ok && passes.next(n, first, count, q)) {
 #define NBOS_PASS(QV)                                                                                 \
     if constexpr (mode_is_ranked(MODE))                                                               \
-        ok = run_pass_ranked<QV, L>(p, smem, stage_bytes, full_bar, empty_bar, abort_flag, ring_pos,  \
+        ok = run_pass_ranked<QV, L, MODE == MODE_RANKED2>(p, smem, stage_bytes, full_bar, empty_bar, abort_flag, ring_pos,  \
                                     tile_begin, tile_end, slice, first, count, n);                    \
     else                                                                                              \
         ok = run_pass<QV, L, MODE>(p, smem, stage_bytes, full_bar, empty_bar, abort_flag, ring_pos,   \
@@ -928,6 +984,7 @@ KernelFn pick_kernel(int mode, int L)
         case MODE_GROUPED: return pick_kernel_l<MODE_GROUPED>(L);
         case MODE_GROUPED2: return pick_kernel_l<MODE_GROUPED2>(L);
         case MODE_RANKED: return pick_kernel_l<MODE_RANKED>(L);
+        case MODE_RANKED2: return pick_kernel_l<MODE_RANKED2>(L);
     }
     return nullptr;
 }
@@ -963,7 +1020,7 @@ int kernel_occupancy(KernelFn fn, int device, size_t smem, int *per_sm)
 int snapshot_mode(const nbos_snapshot *s, int forced)
 {
     if (s->key.key_bits == 64) return MODE_KEY64;
-    if (forced == 0 && s->rank.enabled) return MODE_RANKED;
+    if ((forced == 0 || forced == 5) && s->rank.enabled) return (forced == 0 && s->rank.l1_enabled) ? MODE_RANKED2 : MODE_RANKED;
     if (forced == 1 || !s->pack.enabled) return MODE_PLAIN;
     const bool two = s->pack.guards != s->pack.guards1;
     if ((forced == 0 || forced == 4) && s->key.grouped) return two ? MODE_GROUPED2 : MODE_GROUPED;
@@ -979,6 +1036,7 @@ void fill_params(PlaceParams &p, const nbos_snapshot *s, const int32_t *d_reques
     p.ab = s->d_ab;
     p.pk = s->d_pk;
     p.rk = s->d_rk;
+    p.rk1 = s->d_rk1;
     p.pack = s->pack;
     p.rank = s->rank;
     p.requests = reinterpret_cast<const int4 *>(d_requests);
@@ -1037,7 +1095,7 @@ int make_plan(const nbos_snapshot *s, long long total, long long batch, const nb
     int L = c.lanes_per_request;
     int blocks_per_sm = per_sm;
     {
-        const double pair_cost = (mode_is_sorted(mode) || mode_is_ranked(mode)) ? 3.0 : mode_is_grouped(mode) ? 3.3 : mode_is_static(mode) ? 4.0 : mode_is_packed(mode) ? 5.0
+        const double pair_cost = mode == MODE_RANKED2 ? 2.2 : (mode_is_sorted(mode) || mode_is_ranked(mode)) ? 3.0 : mode_is_grouped(mode) ? 3.3 : mode_is_static(mode) ? 4.0 : mode_is_packed(mode) ? 5.0
                                  : mode == MODE_PLAIN ? 7.0 : 12.0;
         const double kPassCost = 490.0, kRequestCost = 190.0, kHostCost = 1.6, kMergeCost = 12.0;
         const double issue_rate[4] = {0.376, 0.472, 0.499, 0.529};  // per scheduler, by resident blocks
@@ -1114,8 +1172,8 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
         return fail(NBOS_ERR_INVALID_ARG, "requests_per_lane must be 1,2,4 or 8");
     if (c.host_split < 0 || c.grid_blocks < 0 || c.tile_hosts < 0 || (c.tile_hosts & 31))
         return fail(NBOS_ERR_INVALID_ARG, "launch config: negative field or tile_hosts not a multiple of 32");
-    if (c.pair_mode < 0 || c.pair_mode > 4)
-        return fail(NBOS_ERR_INVALID_ARG, "pair_mode must be 0 (automatic), 1 (plain compares), 2 (packed, key computed per pair), 3 (packed, host key compared per pair) or 4 (key-order forms that retire requests)");
+    if (c.pair_mode < 0 || c.pair_mode > 5)
+        return fail(NBOS_ERR_INVALID_ARG, "pair_mode must be 0 (automatic), 1 (plain compares), 2 (packed, key computed per pair), 3 (packed, host key compared per pair), 4 (key-order forms that retire requests) or 5 (ranked form without its first level)");
 
     if (c.first_fit && s->key.static_key && s->presorted) {
         FirstFitParams fp;

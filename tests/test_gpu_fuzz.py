@@ -60,7 +60,7 @@ def test_random_cases(nb, seed):
                  requests_per_lane=int(rng.choice([0, 1, 2, 4, 8])),
                  host_split=int(rng.choice([0, 0, 1, 2, 3])),
                  tile_hosts=int(rng.choice([0, 32, 64, 256])),
-                 pair_mode=int(rng.choice([0, 0, 0, 1, 2, 3, 4])),
+                 pair_mode=int(rng.choice([0, 0, 0, 1, 2, 3, 4, 5])),
                  first_fit=int(rng.choice([0, 0, 1])))
     got = nb.place_workload(w, key_order=key_order, flags=flags | lib_flags, config=nb.launch_config(**shape))
     ref = oracle.place_workload(w, key_order=key_order, flags=flags)

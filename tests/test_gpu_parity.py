@@ -129,7 +129,7 @@ def test_key_widths_orders_flags(nb, lib_flags, key_order, flags):
             assert_same(got, ref, f"{w.name} order={key_order} flags={flags} lib={lib_flags}")
 
 
-@pytest.mark.parametrize("pair_mode", [0, 1, 2, 3, 4])
+@pytest.mark.parametrize("pair_mode", [0, 1, 2, 3, 4, 5])
 @pytest.mark.parametrize("lanes", [0, 1, 4, 32])
 def test_pair_evaluation_modes(nb, pair_mode, lanes):
     """Plain compares, packed test with the key computed or compared per pair, the key-order forms
@@ -194,7 +194,8 @@ def test_ranked_form_coarse_fields(nb):
     resource, with every launch shape; same bytes as the checker."""
     rng = np.random.default_rng(77)
     shapes = (dict(), dict(lanes_per_request=1), dict(lanes_per_request=4, requests_per_lane=2),
-              dict(lanes_per_request=32, tile_hosts=64), dict(lanes_per_request=2, host_split=3, tile_hosts=64))
+              dict(lanes_per_request=32, tile_hosts=64), dict(lanes_per_request=2, host_split=3, tile_hosts=64),
+              dict(pair_mode=5), dict(pair_mode=5, lanes_per_request=8, tile_hosts=96))
     # (a) cfg3-like cluster: millicpus / memory capacities and asks crowd around the same values
     w = W.make_config(3, batch=4000)
     h = w.n_hosts
