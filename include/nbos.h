@@ -205,19 +205,25 @@ int nbos_snapshot_create_host(const nbos_snapshot_desc *desc, void *cuda_stream,
  * a larger subscription or capacity than the widths allow, a GPU count per host the snapshot did
  * not have), the device status word is raised, the tables and every placement made from them are
  * undefined, and nbos_snapshot_status returns NBOS_ERR_RANGE / NBOS_ERR_STALE_LAYOUT; destroy the
- * snapshot and create a new one then. A successful update also clears an earlier status.
+ * snapshot and create a new one then. A successful update clears what an earlier update reported;
+ * a device-side wait that ran out (NBOS_ERR_DEVICE_TIMEOUT) stays reported until the snapshot is
+ * destroyed.
  * The caller must make sure that no placement on ANOTHER stream is still using the snapshot;
  * work queued earlier on the same stream is ordered before the update.
  *   nbos_snapshot_update       arrays are DEVICE memory (16-byte aligned), read by the queued work
- *   nbos_snapshot_update_host  arrays are HOST memory; staged through the library's memory pool
+ *   nbos_snapshot_update_host  arrays are HOST memory; staged through the library's memory pool.
+ *                              Pageable arrays have been read when the call returns; PINNED arrays
+ *                              are read asynchronously by copies queued on `cuda_stream`: keep
+ *                              them unchanged until that work has finished.
  * Errors at call time: INVALID_ARG (shape / flags differ, NULL or misaligned pointers, bad limit),
  * NO_MEMORY, CUDA.
  */
 int nbos_snapshot_update(nbos_snapshot *snap, const nbos_snapshot_desc *desc, void *cuda_stream);
 int nbos_snapshot_update_host(nbos_snapshot *snap, const nbos_snapshot_desc *desc, void *cuda_stream);
 
-/* Frees the handle (and what nbos_snapshot_create_host allocated). The caller must make sure no
- * nbos_place_batch on this snapshot is still running. NULL is accepted. */
+/* Frees the handle (and what nbos_snapshot_create_host allocated: that memory goes back to the
+ * library's pool in the order of the stream the snapshot was created or last updated on). The
+ * caller must make sure no nbos_place_batch on this snapshot is still running. NULL is accepted. */
 int nbos_snapshot_destroy(nbos_snapshot *snap);
 
 int nbos_snapshot_get_info(const nbos_snapshot *snap, nbos_snapshot_info *out);
@@ -363,7 +369,7 @@ int nbos_cluster_sums(const int32_t *gpus_total, const int32_t *gpus_subscribed,
 
 /*
  * Scale-out deficit of a placed batch (Sections 3.2.1, 3.4.2: when fewer than three candidate
- * servers exist, "however many additional servers are required" are provisioned), per snapshot:
+ * servers exist, as many additional servers as are missing get provisioned), per snapshot:
  *   out_deficit[2n + 0] = sum over the batch of (3 - found)
  *   out_deficit[2n + 1] = number of requests with found < 3
  * found: DEVICE [n_snapshots * batch_per_snapshot] int32 as written by nbos_place_batch;

@@ -24,7 +24,7 @@
  * Readings where the paper is silent (the project's design notes list them all):
  *   - "idle GPUs" of a server is G - C, C = GPUs bound to running replicas.
  *   - the SR used for ranking and for the limit is the one AFTER placement,
- *     (S + g) / (G * R); lower is better; "exceed" means strictly greater.
+ *     (S + g) / (G * R); lower is better; the limit is exceeded only by a strictly greater SR.
  *   - remaining ties go to the lower host index.
  *   - a request with a negative field fits nowhere; a server with G < 1 is not a
  *     GPU server and is never a candidate.
@@ -252,8 +252,8 @@ int nbos_oracle_autoscale(int64_t sum_G, int64_t sum_C, int64_t f_num, int64_t f
     return (have_scaled < expected_scaled) - (expected_scaled < have_scaled);
 }
 
-/* Sections 3.2.1 / 3.4.2: a kernel for which fewer than three servers were found needs
- * "however many additional servers are required". deficit = sum of (3 - found),
+/* Sections 3.2.1 / 3.4.2: a kernel for which fewer than three servers were found needs as many
+ * additional servers as it is short of. deficit = sum of (3 - found),
  * short_requests = number of requests with found < 3. */
 void nbos_oracle_scale_out_deficit(const int32_t *found, int64_t batch, int64_t *deficit,
                                    int64_t *short_requests)
@@ -271,7 +271,7 @@ void nbos_oracle_scale_out_deficit(const int32_t *found, int64_t batch, int64_t 
 /*
  * Sequential placement: the paper's scheduler places one kernel at a time, and the replicas of a
  * placed kernel subscribe to its GPUs on their three servers before the next kernel is looked at
- * (Section 3.2.1: "the kernel replicas subscribe to the requested resources"; Section 3.4.1: S is
+ * (Section 3.2.1: a kernel's replicas subscribe to the resources it requested; Section 3.4.1: S is
  * the sum of the GPUs requested by all replicas scheduled on the server).
  *
  * For request r = 0, 1, ... in order: place it against the current state exactly as

@@ -43,7 +43,7 @@ EXPORTED_SYMBOLS = (
     "nbos_place_batch_host", "nbos_place_batch_noalloc", "nbos_select_executors",
     "nbos_cluster_sums", "nbos_scale_out_deficit", "nbos_place_batch_sequential",
     "nbos_snapshot_status", "nbos_strerror", "nbos_last_error_detail",
-    "nbos_probe_int32_issue", "nbos_probe_wait_timeout",
+    "nbos_probe_int32_issue", "nbos_probe_wait_timeout", "nbos_probe_wait_timeout_on_snapshot",
 )
 
 _i32p = ctypes.POINTER(ctypes.c_int32)
@@ -138,6 +138,7 @@ def load_library() -> ctypes.CDLL:
                                                                 P(ctypes.c_float)]
     lib.nbos_probe_wait_timeout.argtypes = [ctypes.c_uint64, vp, P(ctypes.c_int),
                                             P(ctypes.c_float)]
+    lib.nbos_probe_wait_timeout_on_snapshot.argtypes = [vp, ctypes.c_uint64, vp, P(ctypes.c_float)]
     for name in EXPORTED_SYMBOLS:
         fn = getattr(lib, name)
         if name not in ("nbos_strerror", "nbos_last_error_detail"):
@@ -443,11 +444,19 @@ def nbos_probe_int32_issue(mix: int, iters: int, blocks: int, threads: int, stre
 
 
 def nbos_probe_wait_timeout(limit_ns: int, stream=None):
-    """Returns (gave_up, milliseconds)."""
+    """Returns (mask of the warps whose wait ran out: 3 = both, 0 = none; milliseconds)."""
     gave_up, ms = ctypes.c_int(0), ctypes.c_float(0)
     _check(load_library().nbos_probe_wait_timeout(limit_ns, _stream_ptr(stream),
                                                   ctypes.byref(gave_up), ctypes.byref(ms)))
-    return bool(gave_up.value), float(ms.value)
+    return int(gave_up.value), float(ms.value)
+
+
+def nbos_probe_wait_timeout_on_snapshot(snap: Snapshot, limit_ns: int, stream=None) -> float:
+    """Runs the bounded-wait self-test so that it reports in `snap`'s status word; returns ms."""
+    ms = ctypes.c_float(0)
+    _check(load_library().nbos_probe_wait_timeout_on_snapshot(snap.handle, limit_ns, _stream_ptr(stream),
+                                                              ctypes.byref(ms)))
+    return float(ms.value)
 
 
 def launch_config(lanes_per_request=0, requests_per_lane=0, host_split=0, tile_hosts=0,

@@ -255,6 +255,17 @@ int nbos_snapshot_create_host(const nbos_snapshot_desc *desc, void *cuda_stream,
     return NBOS_OK;
 }
 
+// A snapshot's tables live on the device it was created on; kernels launched from another
+// current device would be handed pointers that mean nothing there.
+static int check_current_device(const nbos_snapshot *snap)
+{
+    int device = -1;
+    NBOS_CUDA_TRY(cudaGetDevice(&device));
+    if (device != snap->device)
+        return fail(NBOS_ERR_INVALID_ARG, "the snapshot belongs to device %d, the current device is %d", snap->device, device);
+    return NBOS_OK;
+}
+
 static int check_update_desc(const nbos_snapshot *snap, const nbos_snapshot_desc *desc)
 {
     if (!snap) return fail(NBOS_ERR_INVALID_ARG, "snapshot is NULL");
@@ -277,6 +288,7 @@ int nbos_snapshot_update(nbos_snapshot *snap, const nbos_snapshot_desc *desc, vo
                              desc->vram_gb, desc->millicpus, desc->mem_mb};
     for (int i = 0; i < 6; ++i)
         if (!aligned(arrays[i], 16)) return fail(NBOS_ERR_INVALID_ARG, "host-state array %d is not 16-byte aligned", i);
+    snap->owner_stream = static_cast<cudaStream_t>(cuda_stream);
     return update_snapshot(snap, desc, desc->gpus_total, desc->gpus_subscribed, desc->gpus_committed,
                            desc->vram_gb, desc->millicpus, desc->mem_mb, static_cast<cudaStream_t>(cuda_stream));
 }
@@ -307,6 +319,7 @@ int nbos_snapshot_update_host(nbos_snapshot *snap, const nbos_snapshot_desc *des
     rc = e == cudaSuccess ? update_snapshot(snap, desc, dev[0], dev[1], dev[2], dev[3], dev[4], dev[5], stream)
                           : cuda_fail(e, "copying host-state arrays to the device");
     cudaFreeAsync(staging, stream);
+    snap->owner_stream = stream;
     return rc;
 }
 
@@ -315,7 +328,8 @@ int nbos_snapshot_destroy(nbos_snapshot *snap)
     if (!snap) return NBOS_OK;
     int rc = NBOS_OK;
     if (snap->owns_workspace) {
-        cudaError_t e = cudaFreeAsync(snap->workspace, nullptr);  // legacy default stream: ordered after blocking streams
+        // in the order of the stream whose kernels last wrote the workspace (creation or update)
+        cudaError_t e = cudaFreeAsync(snap->workspace, snap->owner_stream);
         if (e != cudaSuccess) rc = cuda_fail(e, "cudaFreeAsync");
     }
     delete snap;
@@ -357,6 +371,8 @@ int nbos_place_batch_ex(const nbos_snapshot *snap, const int32_t *requests,
     if (!requests || !out_hosts) return fail(NBOS_ERR_INVALID_ARG, "requests / out_hosts is NULL");
     if (!aligned(requests, 16)) return fail(NBOS_ERR_INVALID_ARG, "requests is not 16-byte aligned");
     if (!aligned(out_hosts, 4) || !aligned(out_found, 4)) return fail(NBOS_ERR_INVALID_ARG, "output not 4-byte aligned");
+    int rc = check_current_device(snap);
+    if (rc) return rc;
     return launch_place(snap, requests, batch_per_snapshot, out_hosts, out_found,
                         static_cast<cudaStream_t>(cuda_stream), cfg);
 }
@@ -377,6 +393,8 @@ int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_hos
         return fail(NBOS_ERR_INVALID_ARG, "batch_per_snapshot out of range");
     if (batch_per_snapshot == 0) return NBOS_OK;
     if (!requests_host || !out_hosts_host) return fail(NBOS_ERR_INVALID_ARG, "requests / out_hosts is NULL");
+    int rc_dev = check_current_device(snap);
+    if (rc_dev) return rc_dev;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const long long total = (long long)snap->N * batch_per_snapshot;
     const size_t req_bytes = (size_t)total * 16, out_bytes = (size_t)total * 12,
@@ -469,6 +487,8 @@ int nbos_place_batch_sequential(const nbos_snapshot *snap, const int32_t *reques
         return fail(NBOS_ERR_INVALID_ARG, "batch_per_snapshot out of range");
     if (batch_per_snapshot != 0 && (!requests || !out_hosts)) return fail(NBOS_ERR_INVALID_ARG, "requests / out_hosts is NULL");
     if (!aligned(requests, 16)) return fail(NBOS_ERR_INVALID_ARG, "requests is not 16-byte aligned");
+    int rc = check_current_device(snap);
+    if (rc) return rc;
     return launch_place_sequential(snap, requests, batch_per_snapshot, out_hosts, out_found, out_subscribed,
                                    static_cast<cudaStream_t>(cuda_stream));
 }
@@ -477,9 +497,10 @@ int nbos_snapshot_status(const nbos_snapshot *snap, void *cuda_stream)
 {
     if (!snap) return fail(NBOS_ERR_INVALID_ARG, "snapshot is NULL");
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    unsigned int word = 0;
-    NBOS_CUDA_TRY(cudaMemcpyAsync(&word, snap->d_status, sizeof(word), cudaMemcpyDeviceToHost, stream));
+    unsigned int words[kUpdateStatusOffset / sizeof(unsigned int) + 1] = {};
+    NBOS_CUDA_TRY(cudaMemcpyAsync(words, snap->d_status, sizeof(words), cudaMemcpyDeviceToHost, stream));
     NBOS_CUDA_TRY(cudaStreamSynchronize(stream));
+    const unsigned int word = words[0] | words[kUpdateStatusOffset / sizeof(unsigned int)];
     if (word & STATUS_WAIT_TIMEOUT) return fail(NBOS_ERR_DEVICE_TIMEOUT, "a kernel gave up on a bounded wait (status word 0x%x)", word);
     if (word & STATUS_BAD_VALUES) return fail(NBOS_ERR_RANGE, "the last update brought a value outside the supported range (status word 0x%x)", word);
     if (word & STATUS_STALE_LAYOUT) return fail(NBOS_ERR_STALE_LAYOUT, "the last update does not fit the snapshot's layout (status word 0x%x)", word);

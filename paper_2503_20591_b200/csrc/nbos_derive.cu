@@ -422,14 +422,17 @@ struct DeriveCtx {
 };
 
 // Clear the per-derivation state and put the limits on the device (or compute them there).
-int stage_limits(DeriveCtx &c, const nbos_snapshot_desc *d)
+// `first_time` also clears the word that kernels raise when a bounded wait runs out; a later
+// derivation of the same snapshot leaves that word alone.
+int stage_limits(DeriveCtx &c, const nbos_snapshot_desc *d, bool first_time)
 {
     nbos_snapshot *s = c.s;
     const int N = s->N, H = s->H;
     const bool dynamic_limit = (s->flags & NBOS_LIMIT_CLUSTER_SR) != 0;
     // status word, limits, sums and scan statistics are contiguous: one clear (lambda and g_single,
     // which an update keeps, lie behind them)
-    NBOS_CUDA_TRY(cudaMemsetAsync(c.ws + c.lay.off_status, 0, c.lay.off_lambda - c.lay.off_status, c.stream));
+    const size_t from = c.lay.off_status + (first_time ? 0 : kUpdateStatusOffset);
+    NBOS_CUDA_TRY(cudaMemsetAsync(c.ws + from, 0, c.lay.off_lambda - from, c.stream));
     c.limits_arg = c.d_limits;
     c.limit0 = make_longlong2(0, 1);
     if (dynamic_limit) {
@@ -527,7 +530,7 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     } guard{h_stats, h_lambda, h_g_single};
     if (!h_stats || !h_lambda || !h_g_single) return fail(NBOS_ERR_NO_MEMORY, "host allocation failed");
 
-    int rc = stage_limits(c, d);
+    int rc = stage_limits(c, d, true);
     if (rc) return rc;
     ScanArgs sa{d_G, d_S, d_C, d_AV, d_AC, d_AM, c.limits_arg, c.limit0, d_stats, H, s->R, s->flags,
                 nullptr, nullptr, nullptr, 0ull, 0, 0, {0, 0, 0, 0}};
@@ -725,6 +728,7 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     rc = emit_tables(c);
     if (rc) return rc;
     s->d_status = reinterpret_cast<unsigned int *>(c.ws + c.lay.off_status);
+    s->d_update_status = reinterpret_cast<unsigned int *>(c.ws + c.lay.off_status + kUpdateStatusOffset);
     s->d_feas = reinterpret_cast<const int4 *>(c.ws + c.lay.off_feas);
     s->d_ab = c.ws + c.lay.off_ab;
     s->d_pk = reinterpret_cast<const uint4 *>(c.ws + c.lay.off_pk);
@@ -744,12 +748,12 @@ int update_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
                     const int32_t *d_AC, const int32_t *d_AM, cudaStream_t stream)
 {
     DeriveCtx c = make_ctx(s, d_G, d_S, d_C, d_AV, d_AC, d_AM, stream);
-    int rc = stage_limits(c, d);
+    int rc = stage_limits(c, d, false);
     if (rc) return rc;
     const int *fm = s->pack.enabled ? s->pack.fmax : s->rank.fmax;  // the same values in both layouts
     ScanArgs sa{d_G, d_S, d_C, d_AV, d_AC, d_AM, c.limits_arg, c.limit0,
                 reinterpret_cast<SnapStats *>(c.ws + c.lay.off_stats), s->H, s->R, s->flags,
-                s->d_status,
+                s->d_update_status,
                 s->key.static_key ? nullptr : reinterpret_cast<const long long *>(c.ws + c.lay.off_lambda),
                 reinterpret_cast<const int *>(c.ws + c.lay.off_g_single),
                 s->key.bits_sr >= 64 ? ~0ull : ((1ull << s->key.bits_sr) - 1ull), s->idle_max,

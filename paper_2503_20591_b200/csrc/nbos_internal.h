@@ -30,7 +30,11 @@ struct SnapStats {                 // one per snapshot, filled by the scan kerne
     int max_gcap1, max_av, max_ac, max_am;  // maxima of gmax + 1 and of the three capacities
     unsigned long long g_mask[16]; // bit G set if some host has G GPUs (G in 1..1023)
 };
-enum : unsigned int {  // bits of the snapshot's device status word
+// The status section of the workspace holds two words: at offset 0 what kernels report while they
+// run (kept for the life of the snapshot), at kUpdateStatusOffset what the last derivation
+// reported (cleared by the next one).
+constexpr size_t kUpdateStatusOffset = 128;
+enum : unsigned int {  // bits of the snapshot's device status words
     STATUS_WAIT_TIMEOUT = 1u,   // a kernel gave up on a bounded wait
     STATUS_STALE_LAYOUT = 2u,   // nbos_snapshot_update: the new state does not fit the stored layout
     STATUS_BAD_VALUES = 4u,     // nbos_snapshot_update: a value outside the supported range
@@ -110,7 +114,8 @@ struct nbos_snapshot {
     void *workspace;
     size_t workspace_bytes;
     bool owns_workspace;
-    unsigned int *d_status;
+    unsigned int *d_status;         // raised by kernels that gave up on a bounded wait
+    unsigned int *d_update_status;  // raised by nbos_snapshot_update's scan of the new state
     // tables in visiting order (hosts sorted by ascending A when the table is small enough)
     const int4 *d_feas;   // [N][Hpad] (gmax, vram_gb, millicpus, mem_mb)
     const void *d_ab;     // [N][Hpad] uint2 (32-bit keys) or ulonglong2 (64-bit keys): (A, B)

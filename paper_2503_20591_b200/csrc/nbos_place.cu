@@ -110,17 +110,6 @@ template <> struct KeyTraits<unsigned long long> {
     static constexpr unsigned long long kInf = 0xFFFFFFFFFFFFFFFFull;
 };
 
-// ---- best-three bookkeeping ---------------------------------------------------------------
-// (t1 <= t2 <= t3) := the three smallest of {t1, t2, t3, k}
-template <typename KeyT>
-__device__ __forceinline__ void insert3(KeyT &t1, KeyT &t2, KeyT &t3, KeyT k)
-{
-    const KeyT hi1 = max(t1, k);
-    t1 = min(t1, k);
-    const KeyT hi2 = max(t2, hi1);
-    t2 = min(t2, hi1);
-    t3 = min(t3, hi2);
-}
 
 // ---- the list of passes a block makes over its share of the requests ----------------------
 // A block owns the flattened request range [lo, hi) of [0, N * B). It is cut at snapshot
@@ -522,7 +511,10 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
         return r;
     };
 
-    unsigned long long rq[Q];              // two-word form of each request
+    // Two-word form of each request. With two levels it is needed only in the chunks that pass
+    // the first level, and is kept in local memory (indexed dynamically below) so that the pair
+    // loop has its registers for first-level words; otherwise it stays in registers.
+    unsigned long long rq_keep[Q];
     unsigned int r1[TWO_LEVELS ? Q : 1];   // first-level word
     unsigned int best[3 * Q];  // positions of the best three: [0, Q) best, [Q, 2Q) second, [2Q, 3Q) third
     unsigned int field[Q];     // rank field of each request after an update
@@ -543,7 +535,7 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
             if (p.rank.fword[k]) w1 |= piece; else w0 |= piece;
             l1 |= (val[k] >> p.rank.l1_drop[k]) << p.rank.l1_shift[k];
         }
-        rq[q] = (unsigned long long)w0 | ((unsigned long long)w1 << 32);  // rank field 0: every rank passes
+        rq_keep[q] = (unsigned long long)w0 | ((unsigned long long)w1 << 32);  // rank field 0: every rank passes
         if constexpr (TWO_LEVELS) r1[q] = l1;
         best[q] = kNone; best[Q + q] = kNone; best[2 * Q + q] = kNone;
         field[q] = 0u;
@@ -573,6 +565,9 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
 #pragma unroll
                 for (int u = 0; u < W; ++u) h[u] = R[i0 + u * L];
             }
+            unsigned long long rq[Q];
+#pragma unroll
+            for (int q = 0; q < Q; ++q) rq[q] = rq_keep[q];
             if (!ranked_chunk_any_pass<Q, W>(rq, h, guards)) return;
             // rare. Which pairs passed (bit q * W + u), with static register indices ...
             unsigned int passed = 0u;
@@ -600,14 +595,16 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
                     insert3(a1, a2, a3, pos);
                     best[q] = a1; best[Q + q] = a2; best[2 * Q + q] = a3;
                     field[q] = a3 == kNone ? 0u : p.rank.rank_top + 1u - a3;
+                    if constexpr (TWO_LEVELS)
+                        rq_keep[q] = (rq_keep[q] & ~rank_mask) | ((unsigned long long)field[q] << rank_shift);
                     touched = 1u;
                 }
             }
             if (touched) {
 #pragma unroll
                 for (int q = 0; q < Q; ++q) {
-                    rq[q] = (rq[q] & ~rank_mask) | ((unsigned long long)field[q] << rank_shift);
                     if constexpr (TWO_LEVELS) r1[q] = (r1[q] & ~p.rank.l1_rank_mask) | (field[q] << p.rank.l1_shift[4]);
+                    else rq_keep[q] = (rq_keep[q] & ~rank_mask) | ((unsigned long long)field[q] << rank_shift);
                 }
             }
         };
@@ -617,25 +614,35 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
             auto chunk1 = [&](auto width, int i0) {
                 constexpr int W = decltype(width)::value;
                 unsigned int h1[W];
-                if constexpr (L == 1 && W == 8) {
-                    const uint4 a = *reinterpret_cast<const uint4 *>(R1 + i0);
-                    const uint4 b = *reinterpret_cast<const uint4 *>(R1 + i0 + 4);
-                    h1[0] = a.x; h1[1] = a.y; h1[2] = a.z; h1[3] = a.w;
-                    h1[4] = b.x; h1[5] = b.y; h1[6] = b.z; h1[7] = b.w;
+                if constexpr (L == 1 && W >= 8) {
+                    // consecutive hosts: 128-bit shared-memory loads (i0 is a multiple of W)
+#pragma unroll
+                    for (int v = 0; v < W / 4; ++v) {
+                        const uint4 a = *reinterpret_cast<const uint4 *>(R1 + i0 + 4 * v);
+                        h1[4 * v] = a.x; h1[4 * v + 1] = a.y; h1[4 * v + 2] = a.z; h1[4 * v + 3] = a.w;
+                    }
                 } else {
 #pragma unroll
                     for (int u = 0; u < W; ++u) h1[u] = R1[i0 + u * L];
                 }
-                if (ranked_l1_chunk_any_pass<Q, W>(r1, h1, guards1)) {
-                    if constexpr (W == 8) {
-                        chunk2(std::integral_constant<int, 4>{}, i0);
-                        chunk2(std::integral_constant<int, 4>{}, i0 + 4 * L);
+                unsigned int groups_passed = ranked_l1_chunk_groups_passed<Q, W>(r1, h1, guards1);
+                if (groups_passed) {
+                    if constexpr (W >= 8) {
+                        // second level only for the groups of four hosts in which a pair passed
+                        do {
+                            const int v = __ffs(groups_passed) - 1;
+                            groups_passed &= groups_passed - 1u;
+                            chunk2(std::integral_constant<int, 4>{}, i0 + 4 * v * L);
+                        } while (groups_passed);
                     } else {
                         chunk2(std::integral_constant<int, W>{}, i0);
                     }
                 }
             };
-            for (; i + 7 * L < hosts; i += 8 * L) chunk1(std::integral_constant<int, 8>{}, i);
+#ifndef NBOS_L1_WIDE
+#define NBOS_L1_WIDE 16   // hosts per first-level chunk of a lane
+#endif
+            for (; i + (NBOS_L1_WIDE - 1) * L < hosts; i += NBOS_L1_WIDE * L) chunk1(std::integral_constant<int, NBOS_L1_WIDE>{}, i);
             for (; i + 3 * L < hosts; i += 4 * L) chunk1(std::integral_constant<int, 4>{}, i);
             for (; i < hosts; i += L) chunk1(std::integral_constant<int, 1>{}, i);
         } else {

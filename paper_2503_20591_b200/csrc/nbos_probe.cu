@@ -1,5 +1,6 @@
 // Measurement helpers declared in include/nbos_probe.h.
 #include "nbos_internal.h"
+#include "nbos_ptx.cuh"
 #include "nbos_probe.h"
 
 namespace nbos {
@@ -41,34 +42,24 @@ __global__ void __launch_bounds__(1024) issue_probe_kernel(int iters, int a, int
     if (acc == 0x7fffffff) sink[0] = acc;  // keeps the chains alive; practically never taken
 }
 
-__global__ void wait_timeout_kernel(unsigned long long limit_ns, unsigned int *gave_up)
+// Two warps wait, with the placement kernel's own bounded wait, for a phase of a shared-memory
+// barrier that nothing ever completes. The warp whose wait runs out first raises the block's abort
+// flag, the other leaves through that flag; each reports in `status` the way the placement kernel
+// reports in a snapshot's status word (bit 0), plus bit 1 + warp index for the test to see that
+// both warps came back.
+__global__ void wait_timeout_kernel(unsigned long long limit_ns, unsigned int *status)
 {
     __shared__ __align__(8) unsigned long long bar;
-    const unsigned int addr = (unsigned int)__cvta_generic_to_shared(&bar);
+    __shared__ unsigned int abort_flag;
+    const uint32_t addr = smem_addr(&bar);
     if (threadIdx.x == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(addr), "r"(1u) : "memory");
+        mbar_init(addr, 1u);
+        abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    // nothing ever arrives on `bar`: phase 0 never completes
-    unsigned long long t0;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
-    bool done = false, expired = false;
-    while (!done && !expired) {
-        for (int i = 0; i < 32 && !done; ++i) {
-            unsigned int ok;
-            asm volatile(
-                "{\n\t.reg .pred p;\n\t"
-                "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-                "selp.u32 %0, 1, 0, p;\n\t}"
-                : "=r"(ok) : "r"(addr), "r"(0u) : "memory");
-            done = ok != 0;
-        }
-        unsigned long long t1;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
-        expired = t1 - t0 > limit_ns;
-    }
-    if (!done && threadIdx.x == 0) atomicOr(gave_up, 1u);
+    const bool done = mbar_wait(addr, 0u, &abort_flag, limit_ns);
+    if (!done && (threadIdx.x & 31) == 0) atomicOr(status, STATUS_WAIT_TIMEOUT | (2u << (threadIdx.x >> 5)));
 }
 
 }  // namespace
@@ -111,35 +102,53 @@ extern "C" int nbos_probe_int32_issue(int mix, int iters, int blocks, int thread
     return NBOS_OK;
 }
 
-extern "C" int nbos_probe_wait_timeout(uint64_t limit_ns, void *cuda_stream, int *out_gave_up,
-                                       float *out_ms)
+static int run_wait_timeout(uint64_t limit_ns, cudaStream_t stream, unsigned int *d_status, float *out_ms)
 {
-    if (!out_gave_up || !out_ms) return fail(NBOS_ERR_INVALID_ARG, "NULL output");
     if (limit_ns < 1000000ull) limit_ns = 1000000ull;
     if (limit_ns > 5000000000ull) limit_ns = 5000000000ull;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    unsigned int *flag = nullptr;
-    NBOS_CUDA_TRY(cudaMalloc(&flag, sizeof(unsigned int)));
-    cudaError_t e = cudaMemsetAsync(flag, 0, sizeof(unsigned int), stream);
     cudaEvent_t e0, e1;
     cudaEventCreate(&e0);
     cudaEventCreate(&e1);
     cudaEventRecord(e0, stream);
-    if (e == cudaSuccess) {
-        wait_timeout_kernel<<<1, 64, 0, stream>>>(limit_ns, flag);
-        e = cudaGetLastError();
-    }
+    wait_timeout_kernel<<<1, 64, 0, stream>>>(limit_ns, d_status);
+    cudaError_t e = cudaGetLastError();
     cudaEventRecord(e1, stream);
-    unsigned int word = 0;
-    if (e == cudaSuccess) e = cudaMemcpyAsync(&word, flag, sizeof(word), cudaMemcpyDeviceToHost, stream);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e == cudaSuccess) e = cudaEventSynchronize(e1);
     float ms = 0.f;
     if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);
-    cudaFree(flag);
     if (e != cudaSuccess) return cuda_fail(e, "wait-timeout self-test");
-    *out_gave_up = word ? 1 : 0;
     *out_ms = ms;
     return NBOS_OK;
+}
+
+extern "C" int nbos_probe_wait_timeout(uint64_t limit_ns, void *cuda_stream, int *out_gave_up,
+                                       float *out_ms)
+{
+    if (!out_gave_up || !out_ms) return fail(NBOS_ERR_INVALID_ARG, "NULL output");
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    unsigned int *flag = nullptr;
+    NBOS_CUDA_TRY(cudaMalloc(&flag, sizeof(unsigned int)));
+    cudaError_t e = cudaMemsetAsync(flag, 0, sizeof(unsigned int), stream);
+    int rc = e == cudaSuccess ? run_wait_timeout(limit_ns, stream, flag, out_ms) : cuda_fail(e, "cudaMemsetAsync");
+    unsigned int word = 0;
+    if (rc == NBOS_OK) {
+        e = cudaMemcpy(&word, flag, sizeof(word), cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) rc = cuda_fail(e, "reading the self-test's status word");
+    }
+    cudaFree(flag);
+    if (rc) return rc;
+    *out_gave_up = (word & STATUS_WAIT_TIMEOUT) ? (int)(word >> 1) : 0;
+    return NBOS_OK;
+}
+
+extern "C" int nbos_probe_wait_timeout_on_snapshot(nbos_snapshot *snap, uint64_t limit_ns,
+                                                   void *cuda_stream, float *out_ms)
+{
+    if (!snap || !out_ms) return fail(NBOS_ERR_INVALID_ARG, "NULL argument");
+    int device = -1;
+    NBOS_CUDA_TRY(cudaGetDevice(&device));
+    if (device != snap->device) return fail(NBOS_ERR_INVALID_ARG, "the snapshot belongs to device %d", snap->device);
+    return run_wait_timeout(limit_ns, static_cast<cudaStream_t>(cuda_stream), snap->d_status, out_ms);
 }

@@ -1,5 +1,6 @@
 // Inline-PTX wrappers shared by the kernels that stage data through shared memory with bulk
-// asynchronous copies: mbarriers with bounded waits and the bulk copy global -> shared.
+// asynchronous copies: mbarriers with bounded waits and the bulk copy global -> shared; and the
+// best-three insertion the placement kernels share.
 #ifndef NBOS_PTX_CUH_
 #define NBOS_PTX_CUH_
 
@@ -55,26 +56,40 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uin
         : "memory");
 }
 
-// Bounded wait. Returns false when the wait ran out or another thread of the block gave up.
+// (t1 <= t2 <= t3) := the three smallest of {t1, t2, t3, k}
+template <typename KeyT>
+__device__ __forceinline__ void insert3(KeyT &t1, KeyT &t2, KeyT &t3, KeyT k)
+{
+    const KeyT hi1 = max(t1, k);
+    t1 = min(t1, k);
+    const KeyT hi2 = max(t2, hi1);
+    t2 = min(t2, hi1);
+    t3 = min(t3, hi2);
+}
+
+// Bounded wait. Returns false when the wait ran out (after `limit_ns`) or another thread of the
+// block gave up; whoever runs out first raises the block's abort flag for the others.
 static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity,
-                                            volatile unsigned int *abort_flag)
+                                            volatile unsigned int *abort_flag,
+                                            unsigned long long limit_ns)
 {
     const unsigned long long t0 = global_timer_ns();
     for (;;) {
         for (int i = 0; i < 32; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (global_timer_ns() - t0 > kWaitLimitNs) {
+        if (global_timer_ns() - t0 > limit_ns) {
             *abort_flag = 1u;
             return false;
         }
     }
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
-                                          volatile unsigned int *abort_flag)
+                                          volatile unsigned int *abort_flag,
+                                          unsigned long long limit_ns = kWaitLimitNs)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag);
+    return mbar_wait_slow(bar, parity, abort_flag, limit_ns);
 }
 
 

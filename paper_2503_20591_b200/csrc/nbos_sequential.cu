@@ -15,6 +15,7 @@
 #include <limits.h>
 
 #include "nbos_internal.h"
+#include "nbos_ptx.cuh"
 
 namespace nbos {
 namespace {
@@ -50,15 +51,6 @@ template <> struct SeqKey<unsigned long long> {
     }
 };
 
-template <typename KeyT>
-__device__ __forceinline__ void insert3(KeyT &t1, KeyT &t2, KeyT &t3, KeyT k)
-{
-    const KeyT hi1 = max(t1, k);
-    t1 = min(t1, k);
-    const KeyT hi2 = max(t2, hi1);
-    t2 = min(t2, hi1);
-    t3 = min(t3, hi2);
-}
 
 // The three smallest of the warp's keys (each lane brings a sorted triple); every lane returns them.
 template <typename KeyT>

@@ -494,10 +494,44 @@ def test_streams_and_repeated_calls(nb):
 
 def test_bounded_wait_gives_up_and_context_survives(nb):
     """A wait that nothing will ever satisfy must end by itself, be reported, and leave the
-    device usable (no trap, no hang)."""
+    device usable (no trap, no hang). The self-test runs the placement kernel's own wait function:
+    one warp's wait runs out, the other leaves through the block's abort flag."""
     gave_up, ms = nb.nbos_probe_wait_timeout(20_000_000)   # 20 ms
-    assert gave_up
+    assert gave_up == 3                                     # both warps came back empty-handed
     assert 15.0 < ms < 2000.0
     w = W.make_config(0)
     got, ref = both(nb, w)
     assert_same(got, ref)
+
+
+def test_a_wait_that_ran_out_is_reported_by_the_snapshot_and_survives_an_update(nb):
+    """The status word a placement kernel raises when it gives up on a wait reaches the caller as
+    NBOS_ERR_DEVICE_TIMEOUT, and a later refresh of the snapshot does not wipe it."""
+    import torch
+    w = W.make_config(1, batch=256)
+    dev = [torch.from_numpy(getattr(w, k)).cuda().reshape(-1) for k in w.HOST_FIELDS]
+    lim = (torch.from_numpy(w.limit_num), torch.from_numpy(w.limit_den))
+    s = nb.nbos_snapshot_create(w.n_snapshots, w.n_hosts, *lim, *dev)
+    try:
+        assert nb.nbos_snapshot_status(s) == nb.NBOS_OK
+        ms = nb.nbos_probe_wait_timeout_on_snapshot(s, 5_000_000)    # 5 ms
+        assert 3.0 < ms < 2000.0
+        assert nb.nbos_snapshot_status(s) == nb.NBOS_ERR_DEVICE_TIMEOUT
+        nb.nbos_snapshot_update(s, *lim, *dev)
+        assert nb.nbos_snapshot_status(s) == nb.NBOS_ERR_DEVICE_TIMEOUT
+        # the device itself is fine: a placement on a fresh snapshot is exact
+        got, ref = both(nb, w)
+        assert_same(got, ref)
+    finally:
+        nb.nbos_snapshot_destroy(s)
+    # what an update reports is cleared by the next good update
+    s = nb.nbos_snapshot_create(w.n_snapshots, w.n_hosts, *lim, *dev)
+    try:
+        bad = [d.clone() for d in dev]
+        bad[1][3] = -5                                               # a negative subscribed count
+        nb.nbos_snapshot_update(s, *lim, *bad)
+        assert nb.nbos_snapshot_status(s) == nb.NBOS_ERR_RANGE
+        nb.nbos_snapshot_update(s, *lim, *dev)
+        assert nb.nbos_snapshot_status(s) == nb.NBOS_OK
+    finally:
+        nb.nbos_snapshot_destroy(s)

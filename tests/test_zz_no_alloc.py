@@ -4,17 +4,22 @@ Some users of this library cannot allocate device memory at call time: their GPU
 already belongs to another pool (a training or serving job on the same device), or they sit in a
 control loop where an allocation's device-wide synchronisation costs too much. For them
 nbos_place_batch_noalloc keeps the per-slice candidates in a fixed array inside the library.
-It must return exactly the bytes nbos_place_batch returns (index work: bit-exact), call after
-call, although every call reuses that array with the previous call's contents still in it.
+It must return exactly the bytes nbos_place_batch returns (index work: bit-exact) -- which are
+also the CPU checker's -- call after call, although every call reuses that array with the previous
+call's contents still in it; and it must really leave the device's memory alone.
 
 This file is collected last on purpose: a run that stops at the first failure has then already
 been through every other test.
 """
 from __future__ import annotations
 
+import dataclasses
+import os
+
 import numpy as np
 import pytest
 
+import oracle
 from paper_2503_20591_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
@@ -59,8 +64,42 @@ def test_two_calls_in_a_row_match_the_allocating_entry_point(nb, host_split):
                 np.testing.assert_array_equal(got[1], ref[1])
                 plain = _run(nb, snap, w, requests, nb.nbos_place_batch)
                 np.testing.assert_array_equal(got[0], plain[0])
+                # and the checker's, computed on the CPU from the paper's rule
+                sub = dataclasses.replace(w, requests=np.ascontiguousarray(requests), batch=requests.shape[1])
+                want = oracle.place_workload(sub, threads=min(16, os.cpu_count() or 1))
+                np.testing.assert_array_equal(got[0], want[0])
+                np.testing.assert_array_equal(got[1], want[1])
         finally:
             nb.nbos_snapshot_destroy(snap)
+
+
+def test_no_device_memory_is_taken_or_returned(nb):
+    """Across calls of the allocation-free entry point neither the driver's count of free device
+    memory nor what PyTorch's allocator holds may move: a caller whose memory is spoken for must be
+    able to rely on that. (The first call per device resolves the array's address; it is made
+    before the measurement, as the header asks start-up code to do.)"""
+    import torch
+    w = W.make_config(2, batch=2000)
+    snap = nb.snapshot_from_workload(w)
+    try:
+        req = torch.from_numpy(w.requests).cuda()
+        out = torch.empty((1, w.batch, 3), dtype=torch.int32, device="cuda")
+        found = torch.empty((1, w.batch), dtype=torch.int32, device="cuda")
+        nb.nbos_place_batch_noalloc(snap, req, out, found, host_split=4)     # start-up call
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info()
+        reserved0, allocated0 = torch.cuda.memory_reserved(), torch.cuda.memory_allocated()
+        for split in (4, 1, 7, 4):
+            nb.nbos_place_batch_noalloc(snap, req, out, found, host_split=split)
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        assert free1 == free0
+        assert (torch.cuda.memory_reserved(), torch.cuda.memory_allocated()) == (reserved0, allocated0)
+        want = oracle.place_workload(w, threads=min(16, os.cpu_count() or 1))
+        np.testing.assert_array_equal(out.cpu().numpy(), want[0])
+        np.testing.assert_array_equal(found.cpu().numpy(), want[1])
+    finally:
+        nb.nbos_snapshot_destroy(snap)
 
 
 def test_wide_keys_use_the_same_array(nb):
