@@ -49,7 +49,8 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
-    ap.add_argument("--workload", type=int, default=3, help="benchmark workload index 0..4")
+    ap.add_argument("--workload", type=int, default=3,
+                    help="benchmark workload index 0..4; 5 = 4,096 servers with 1..8 GPUs (not one of the five)")
     ap.add_argument("--batch", type=int, default=None, help="shrink the batch (profiling captures)")
     ap.add_argument("--snapshots", type=int, default=None, help="shrink workload 4")
     ap.add_argument("--min-timed-ms", type=float, default=1000.0,
@@ -161,12 +162,18 @@ def time_checker(w, sample: int, steps: int, warmup: int):
     return w.n_snapshots * min(sample, w.batch), dt, res
 
 
+def make_workload(W, args):
+    if args.workload == 5:
+        return W.mixed_gpu_cluster(4096, args.batch or (1 << 20), seed=5, name="mixed_gpu_counts_4096")
+    return W.make_config(args.workload, batch=args.batch, n_snapshots=args.snapshots)
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
     from paper_2503_20591_b200 import workloads as W
-    w = W.make_config(args.workload, batch=args.batch, n_snapshots=args.snapshots)
+    w = make_workload(W, args)
     # size the sample so that the whole run stays near a minute at ~25 M pairs/s per core
     budget_pairs = 60.0 * 25e6 / max(1, args.steps + args.warmup)
     sample = args.cpu_sample or int(budget_pairs / (w.n_snapshots * w.n_hosts))
@@ -301,7 +308,7 @@ def run_ours(args):
     # total exceeds the L2 cache. Weak scaling: every rank places its own full batch. Strong
     # scaling: the same batches on every rank, each rank places its slice of the flattened
     # request list (single-snapshot workloads) ----
-    w = W.make_config(args.workload, batch=args.batch, n_snapshots=args.snapshots)
+    w = make_workload(W, args)
     strong = args.scaling == "strong" and world > 1
     if strong and w.n_snapshots != 1:
         raise SystemExit("--scaling strong cuts the batch of a single-snapshot workload")
@@ -309,8 +316,12 @@ def run_ours(args):
     n_rot = max(2, min(12, -(-int(1.3 * L2_BYTES) // per_batch_bytes)))
     own_first = rank == 0 or strong
     batches = [w.requests] if own_first else []
-    batches += W.extra_request_batches(args.workload, n_rot - len(batches), batch=w.batch,
-                                       n_snapshots=w.n_snapshots, seed0=10_000 + (0 if strong else 1000 * rank))
+    if args.workload == 5:
+        batches += [W.mixed_gpu_cluster(w.n_hosts, w.batch, seed=50 + k + (0 if strong else 100 * rank)).requests
+                    for k in range(n_rot - len(batches))]
+    else:
+        batches += W.extra_request_batches(args.workload, n_rot - len(batches), batch=w.batch,
+                                           n_snapshots=w.n_snapshots, seed0=10_000 + (0 if strong else 1000 * rank))
     lo, hi = sharding.shard_bounds(w.batch, rank, world) if strong else (0, w.batch)
     my_batch = hi - lo
     d_state = [torch.from_numpy(getattr(w, k)).to(dev).reshape(-1) for k in w.HOST_FIELDS]
@@ -568,8 +579,8 @@ def run_ours(args):
         others = {}
         shapes = [W.make_config(idx) for idx in range(5) if idx != args.workload or args.batch is not None]
         # not one of the five: servers with 1..8 GPUs, so that the ranking depends on the ask
-        if args.all_workloads:
-            shapes.append(W.mixed_gpu_cluster(4096, 1 << 20, seed=5, name="mixed_gpu_counts_4096x1M"))
+        if args.all_workloads and args.workload != 5:
+            shapes.append(W.mixed_gpu_cluster(4096, 1 << 20, seed=5, name="mixed_gpu_counts_4096"))
         for ww in shapes:
             sn = nb.snapshot_from_workload(ww, device=dev)
             rq = torch.from_numpy(ww.requests).to(dev)

@@ -1102,10 +1102,17 @@ int make_plan(const nbos_snapshot *s, long long total, long long batch, const nb
     int L = c.lanes_per_request;
     int blocks_per_sm = per_sm;
     {
-        const double pair_cost = mode == MODE_RANKED2 ? 2.2 : (mode_is_sorted(mode) || mode_is_ranked(mode)) ? 3.0 : mode_is_grouped(mode) ? 3.3 : mode_is_static(mode) ? 4.0 : mode_is_packed(mode) ? 5.0
-                                 : mode == MODE_PLAIN ? 7.0 : 12.0;
-        const double kPassCost = 490.0, kRequestCost = 190.0, kHostCost = 1.6, kMergeCost = 12.0;
-        const double issue_rate[4] = {0.376, 0.472, 0.499, 0.529};  // per scheduler, by resident blocks
+        const bool two_level = mode == MODE_RANKED2;
+        const double pair_cost = two_level ? 1.8 : (mode_is_sorted(mode) || mode_is_ranked(mode)) ? 3.0 : mode_is_grouped(mode) ? 3.3
+                                 : mode_is_static(mode) ? 4.0 : mode_is_packed(mode) ? 5.0 : mode == MODE_PLAIN ? 7.0 : 12.0;
+        // The two-level ranked form has a cheap pair step and a dearer start of every request (its
+        // first hosts go through the second level and the exact test until the best three are
+        // full); its constants were fitted on their own.
+        const double kPassCost = two_level ? 3000.0 : 490.0, kRequestCost = two_level ? 930.0 : 190.0,
+                     kHostCost = two_level ? 1.7 : 1.6, kMergeCost = 12.0;
+        const double issue_rate_general[4] = {0.376, 0.472, 0.499, 0.529};  // per scheduler, by resident blocks
+        const double issue_rate_two_level[4] = {0.543, 0.654, 0.774, 0.835};
+        const double *issue_rate = two_level ? issue_rate_two_level : issue_rate_general;
         const long long B = batch > 0 ? batch : total;
         double best = 0.0;
         bool have = false;
