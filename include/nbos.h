@@ -250,10 +250,12 @@ int nbos_place_batch_ex(const nbos_snapshot *snap, const int32_t *requests,
 
 /*
  * Same operation with HOST buffers (pinned memory makes the copies asynchronous and faster, but
- * any host memory works). The batch is cut into up to 8 chunks whose host-to-device copy, kernel
+ * any host memory works). The batch is cut into up to 4 chunks whose host-to-device copy, kernel
  * and device-to-host copy overlap on three internal streams (created once per device; calls on
- * the same device take turns). Device staging comes from the library's own memory pool. Returns
- * after the results are in the host buffers.
+ * the same device take turns). The copies in start at once; the kernels wait for the work queued
+ * on `cuda_stream` before the call (a snapshot update, say). Device staging is a buffer the library
+ * keeps per device and grows when a larger batch comes. Returns after the results are in the host
+ * buffers.
  */
 int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_host,
                           int64_t batch_per_snapshot, int32_t *out_hosts_host,

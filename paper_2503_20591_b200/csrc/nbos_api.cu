@@ -91,6 +91,11 @@ struct HostPipe {
     // unlimited, so the buffers of one call are reused by the next instead of going back to the
     // driver at every synchronisation (which costs more than the placement itself).
     cudaMemPool_t pool = nullptr;
+    // Device staging of nbos_place_batch_host (requests in, results out), kept between calls and
+    // grown when a larger batch comes: calls on a device take turns and each ends synchronised,
+    // so the buffer is free again when the next call starts.
+    char *stage = nullptr;
+    size_t stage_bytes = 0;
 };
 HostPipe g_pipes[64];
 std::mutex g_pipes_mutex;
@@ -407,48 +412,64 @@ int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_hos
     if (rc) return rc;
     std::lock_guard<std::mutex> lock(pipe->mutex);
 
-    char *buf = nullptr;
-    cudaError_t e = cudaMallocFromPoolAsync(reinterpret_cast<void **>(&buf), up(req_bytes) + up(out_bytes) + up(found_bytes), pipe->pool, stream);
-    if (e != cudaSuccess) {
-        cudaGetLastError();
-        return fail(NBOS_ERR_NO_MEMORY, "device staging allocation failed: %s", cudaGetErrorString(e));
+    const size_t need = up(req_bytes) + up(out_bytes) + up(found_bytes);
+    if (pipe->stage_bytes < need) {
+        if (pipe->stage) cudaFree(pipe->stage);
+        pipe->stage = nullptr;
+        pipe->stage_bytes = 0;
+        cudaError_t ea = cudaMalloc(reinterpret_cast<void **>(&pipe->stage), need);
+        if (ea != cudaSuccess) {
+            cudaGetLastError();
+            return fail(NBOS_ERR_NO_MEMORY, "device staging allocation of %zu bytes failed: %s", need, cudaGetErrorString(ea));
+        }
+        pipe->stage_bytes = need;
     }
+    char *buf = pipe->stage;
     int32_t *d_req = reinterpret_cast<int32_t *>(buf);
     int32_t *d_out = reinterpret_cast<int32_t *>(buf + up(req_bytes));
     int32_t *d_found = out_found_host ? reinterpret_cast<int32_t *>(buf + up(req_bytes) + up(out_bytes)) : nullptr;
 
     // chunks of the flattened request list: copy in, place, copy out, round-robin over the side
     // streams so that the copies of one chunk overlap the kernel of another. A chunk carries at
-    // least 2^28 (request, host) pairs (some 40 us of placement), so that the kernel keeps the
-    // efficiency of a large launch; at most eight chunks. Every chunk launch plans itself.
+    // least 2^30 (request, host) pairs: smaller launches lose more in kernel efficiency than the
+    // finer overlap gains (measured with 2, 4, 8, 16 and 32 chunks of the largest benchmark
+    // shape: 0.73, 0.68, 0.69, 0.78, 1.03 ms per call); at most four chunks. Every chunk launch
+    // plans itself. The copies in do not depend on anything queued on the caller's stream (the
+    // staging buffer is this call's alone) and start at once; only the kernels wait for it,
+    // because the snapshot may still be in the making there.
     const long long pairs = total * (long long)snap->Hpad;
-    long long n_chunks = pairs >> 28;
+    long long n_chunks = pairs >> 30;
     if (n_chunks < 1) n_chunks = 1;
-    if (n_chunks > 8) n_chunks = 8;
+    if (n_chunks > 4) n_chunks = 4;
     const long long chunk = (((total + n_chunks - 1) / n_chunks) + 31) & ~31ll;
-    e = cudaEventRecord(pipe->start, stream);
-    for (int j = 0; j < HostPipe::kStreams && e == cudaSuccess; ++j) e = cudaStreamWaitEvent(pipe->streams[j], pipe->start, 0);
+    cudaError_t e = cudaEventRecord(pipe->start, stream);
+    bool waited[HostPipe::kStreams] = {};
     int used = 0;
     for (long long lo = 0, i = 0; lo < total && e == cudaSuccess && rc == NBOS_OK; lo += chunk, ++i) {
         const long long n = total - lo < chunk ? total - lo : chunk;
-        cudaStream_t st = pipe->streams[i % HostPipe::kStreams];
+        const int j = (int)(i % HostPipe::kStreams);
+        cudaStream_t st = pipe->streams[j];
         if (i < HostPipe::kStreams) used = (int)i + 1;
         e = cudaMemcpyAsync(d_req + lo * 4, requests_host + lo * 4, (size_t)n * 16, cudaMemcpyHostToDevice, st);
         if (e != cudaSuccess) break;
+        if (!waited[j]) {
+            e = cudaStreamWaitEvent(st, pipe->start, 0);
+            if (e != cudaSuccess) break;
+            waited[j] = true;
+        }
         rc = launch_place(snap, d_req, batch_per_snapshot, d_out, d_found, st, nullptr, lo, n);
         if (rc) break;
         e = cudaMemcpyAsync(out_hosts_host + lo * 3, d_out + lo * 3, (size_t)n * 12, cudaMemcpyDeviceToHost, st);
         if (e == cudaSuccess && d_found)
             e = cudaMemcpyAsync(out_found_host + lo, d_found + lo, (size_t)n * 4, cudaMemcpyDeviceToHost, st);
     }
-    // join the side streams back into the caller's stream (also on the error paths, so that the
-    // staging buffer is not released under work that was already queued)
+    // join the side streams back into the caller's stream (also on the error paths, so that
+    // nothing of this call is still queued when the next one reuses the staging buffer)
     for (int j = 0; j < used; ++j) {
         cudaError_t e3 = cudaEventRecord(pipe->done[j], pipe->streams[j]);
         if (e3 == cudaSuccess) e3 = cudaStreamWaitEvent(stream, pipe->done[j], 0);
         if (e3 != cudaSuccess && e == cudaSuccess) e = e3;
     }
-    cudaFreeAsync(buf, stream);
     cudaError_t e2 = cudaStreamSynchronize(stream);
     if (rc) return rc;
     if (e != cudaSuccess) return cuda_fail(e, "host <-> device copy");
