@@ -96,6 +96,7 @@ struct PlaceParams {
     long long first_req, n_req;  // this launch handles flattened requests [first_req, first_req + n_req)
     int N, Hpad;
     int tile_hosts, tiles_total, K, req_ctas;
+    int per_snapshot;       // > 0: blocks do not share snapshots, each snapshot's requests go to this many blocks
     unsigned int id_mask;
     int max_q;
 };
@@ -141,6 +142,18 @@ struct PassList {
 __device__ __forceinline__ void block_request_range(const PlaceParams &p, int cr, long long &lo,
                                                     long long &hi)
 {
+    if (p.per_snapshot > 0) {
+        // snapshot cr / per_snapshot, part cr % per_snapshot of its requests (units of 32)
+        const long long n = cr / p.per_snapshot, part = cr % p.per_snapshot;
+        const long long units_b = (p.B + 31) >> 5;
+        lo = (units_b * part / p.per_snapshot) << 5;
+        hi = (units_b * (part + 1) / p.per_snapshot) << 5;
+        if (lo > p.B) lo = p.B;
+        if (hi > p.B) hi = p.B;
+        lo += n * p.B;
+        hi += n * p.B;
+        return;
+    }
     // split in units of 32 requests so that a warp's 128-bit loads start on a 512-byte line
     const long long units = (p.n_req + 31) >> 5;
     lo = (units * cr / p.req_ctas) << 5;
@@ -478,11 +491,26 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
 // ---- one pass in ranked form ------------------------------------------------------------------
 // Same contract as run_pass. The best three of a request are kept as positions in the table
 // (which is stored in key order, so a smaller position is a smaller key) and turned into keys
-// after the last tile. Per pair: one subtraction and one logic operation on the first-level
-// words (TWO_LEVELS), or directly the two-word test. A chunk in which some pair passed the first
-// level goes through the two-word test; pairs that pass that one too are re-tested with the exact
-// records (four compares against the request as it was given), fitting hosts enter the best
-// three, and the request's rank fields are set from its new third best.
+// after the last tile.
+//
+// Hosts are dealt to the L lanes of a request group in groups of four consecutive hosts (lane s
+// takes groups s, s + L, ...), so that a lane's host words come in 128-bit shared-memory loads
+// whatever L is.
+//
+// Opening. The first 16 hosts of the block's slice of the table are compared exactly (four
+// compares on the exact records) against every request of the pass, in table order, until a
+// request has three hosts: in a table in key order most requests find their three right there,
+// and the pair loop then starts with the rank thresholds already in the request words instead
+// of going through the second level and the exact test for its first chunks. Every lane of a
+// group does this (they all need the thresholds); lane 0 of the group keeps the finds.
+//
+// Pair loop, from host 16 on. Per pair: one subtraction and one logic operation on the
+// first-level words (TWO_LEVELS), or directly the two-word test. A group of four hosts in which
+// some pair passed the first level goes through the two-word test; pairs that pass that one too
+// are re-tested with the exact records, fitting hosts enter the best three, and the request's
+// rank fields are set from its new third best (or from the opening's, whichever is earlier).
+constexpr int kOpeningHosts = 16;
+
 template <int Q, int L, bool TWO_LEVELS>
 __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned char *stages,
                                                 uint32_t stage_bytes, uint32_t full_bar,
@@ -501,6 +529,7 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
     const unsigned int guards1 = p.rank.l1_guards;
     const int rank_shift = p.rank.fshift[4] + 32 * p.rank.fword[4];
     const unsigned long long rank_mask = (unsigned long long)p.rank.rank_mask << (32 * p.rank.fword[4]);
+    const int T = p.tile_hosts;
 
     // the ask as given, with a GPU count no host has when it fits nowhere (negative field)
     auto load_request = [&](int q) -> int4 {
@@ -518,9 +547,44 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
     unsigned int r1[TWO_LEVELS ? Q : 1];   // first-level word
     unsigned int best[3 * Q];  // positions of the best three: [0, Q) best, [Q, 2Q) second, [2Q, 3Q) third
     unsigned int field[Q];     // rank field of each request after an update
+    unsigned int opened[Q];    // position of the third host the opening found (kNone: fewer than three)
+
+    // ---- opening: the first hosts of the slice, exactly, eight at a time ----
+    const int open_pos = tile_begin * T;
+    unsigned int o1[Q], o2[Q], o3[Q];
+    int4 ask[Q];
 #pragma unroll
     for (int q = 0; q < Q; ++q) {
-        const int4 r = load_request(q);
+        ask[q] = load_request(q);
+        o1[q] = kNone; o2[q] = kNone; o3[q] = kNone;
+    }
+#pragma unroll 1
+    for (int base = 0; base < kOpeningHosts; base += 8) {
+        bool need = false;
+#pragma unroll
+        for (int q = 0; q < Q; ++q) need |= o3[q] == kNone;
+        if (!need) break;
+        int4 f[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) f[u] = __ldg(p.feas + row + open_pos + base + u);
+#pragma unroll
+        for (int q = 0; q < Q; ++q)
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const bool ok = (ask[q].x <= f[u].x) & (ask[q].y <= f[u].y) & (ask[q].z <= f[u].z) & (ask[q].w <= f[u].w);
+                // positions come in ascending order: a fitting host takes the first free slot
+                const unsigned int pos = (unsigned int)(open_pos + base + u);
+                const bool take3 = ok & (o2[q] != kNone) & (o3[q] == kNone);
+                const bool take2 = ok & (o1[q] != kNone) & (o2[q] == kNone);
+                const bool take1 = ok & (o1[q] == kNone);
+                o3[q] = take3 ? pos : o3[q];
+                o2[q] = take2 ? pos : o2[q];
+                o1[q] = take1 ? pos : o1[q];
+            }
+    }
+#pragma unroll
+    for (int q = 0; q < Q; ++q) {
+        const int4 r = ask[q];
         // an ask above every host's capacity in some resource fits nowhere either: encode both
         // cases as a GPU ask above every gmax and keep the other fields inside their widths
         const bool bad = (r.x > p.rank.fmax[0]) | (r.y > p.rank.fmax[1]) | (r.z > p.rank.fmax[2]) |
@@ -535,13 +599,16 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
             if (p.rank.fword[k]) w1 |= piece; else w0 |= piece;
             l1 |= (val[k] >> p.rank.l1_drop[k]) << p.rank.l1_shift[k];
         }
-        rq_keep[q] = (unsigned long long)w0 | ((unsigned long long)w1 << 32);  // rank field 0: every rank passes
-        if constexpr (TWO_LEVELS) r1[q] = l1;
-        best[q] = kNone; best[Q + q] = kNone; best[2 * Q + q] = kNone;
-        field[q] = 0u;
+        // rank field from the opening's third host (0 = every rank passes)
+        const unsigned int fld = o3[q] == kNone ? 0u : p.rank.rank_top + 1u - o3[q];
+        rq_keep[q] = ((unsigned long long)w0 | ((unsigned long long)w1 << 32)) | ((unsigned long long)fld << rank_shift);
+        if constexpr (TWO_LEVELS) r1[q] = l1 | (fld << p.rank.l1_shift[4]);
+        const bool keeper = sub == 0;   // one lane of the group carries the opening's finds to the merge
+        best[q] = keeper ? o1[q] : kNone; best[Q + q] = keeper ? o2[q] : kNone; best[2 * Q + q] = keeper ? o3[q] : kNone;
+        field[q] = fld;
+        opened[q] = o3[q];
     }
 
-    const int T = p.tile_hosts;
     for (int t = tile_begin; t < tile_end; ++t, ++ring_pos) {
         const uint32_t s = ring_pos % kStages;
         const uint32_t parity = (ring_pos / kStages) & 1u;
@@ -551,33 +618,30 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
         const int pos0 = t * T;
         int hosts = p.Hpad - pos0;
         if (hosts > T) hosts = T;
+        const int n_groups = hosts >> 2;   // groups of four hosts in this tile (hosts is a multiple of 32)
 
-        // two-word test of W hosts (i0, i0 + L, ...) against the Q requests, then the exact part
-        auto chunk2 = [&](auto width, int i0) {
-            constexpr int W = decltype(width)::value;
-            unsigned long long h[W];
-            if constexpr (L == 1 && W == 4) {
-                // consecutive hosts: two 128-bit shared-memory loads (i0 is a multiple of 4)
-                const ulonglong2 a = *reinterpret_cast<const ulonglong2 *>(R + i0);
-                const ulonglong2 b = *reinterpret_cast<const ulonglong2 *>(R + i0 + 2);
+        // two-word test of host group gi (hosts 4 gi .. 4 gi + 3 of the tile) against the Q
+        // requests, then the exact part
+        auto group2 = [&](int gi) {
+            unsigned long long h[4];
+            {
+                const ulonglong2 a = *reinterpret_cast<const ulonglong2 *>(R + 4 * gi);
+                const ulonglong2 b = *reinterpret_cast<const ulonglong2 *>(R + 4 * gi + 2);
                 h[0] = a.x; h[1] = a.y; h[2] = b.x; h[3] = b.y;
-            } else {
-#pragma unroll
-                for (int u = 0; u < W; ++u) h[u] = R[i0 + u * L];
             }
             unsigned long long rq[Q];
 #pragma unroll
             for (int q = 0; q < Q; ++q) rq[q] = rq_keep[q];
-            if (!ranked_chunk_any_pass<Q, W>(rq, h, guards)) return;
-            // rare. Which pairs passed (bit q * W + u), with static register indices ...
+            if (!ranked_chunk_any_pass<Q, 4>(rq, h, guards)) return;
+            // rare. Which pairs passed (bit 4 q + u), with static register indices ...
             unsigned int passed = 0u;
 #pragma unroll
             for (int q = 0; q < Q; ++q)
 #pragma unroll
-                for (int u = 0; u < W; ++u) {
+                for (int u = 0; u < 4; ++u) {
                     const unsigned long long d = h[u] - rq[q];
                     const unsigned int fell = ~((unsigned int)d & (unsigned int)(d >> 32)) & guards;
-                    passed |= (fell == 0u ? 1u : 0u) << (q * W + u);
+                    passed |= (fell == 0u ? 1u : 0u) << (q * 4 + u);
                 }
             // ... then one pair after the other: exact test against the request as given; the
             // best-three arrays are indexed dynamically here and therefore live in local memory,
@@ -586,15 +650,16 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
             while (passed) {
                 const int bit = __ffs(passed) - 1;
                 passed &= passed - 1u;
-                const int q = bit / W, u = bit % W;
-                const unsigned int pos = (unsigned int)(pos0 + i0 + u * L);
+                const int q = bit >> 2, u = bit & 3;
+                const unsigned int pos = (unsigned int)(pos0 + 4 * gi + u);
                 const int4 r = load_request(q);
                 const int4 f = __ldg(p.feas + row + pos);
                 if ((r.x <= f.x) & (r.y <= f.y) & (r.z <= f.z) & (r.w <= f.w)) {
                     unsigned int a1 = best[q], a2 = best[Q + q], a3 = best[2 * Q + q];
                     insert3(a1, a2, a3, pos);
                     best[q] = a1; best[Q + q] = a2; best[2 * Q + q] = a3;
-                    field[q] = a3 == kNone ? 0u : p.rank.rank_top + 1u - a3;
+                    const unsigned int third = min(a3, opened[q]);   // the other lanes' opening finds count too
+                    field[q] = third == kNone ? 0u : p.rank.rank_top + 1u - third;
                     if constexpr (TWO_LEVELS)
                         rq_keep[q] = (rq_keep[q] & ~rank_mask) | ((unsigned long long)field[q] << rank_shift);
                     touched = 1u;
@@ -609,45 +674,32 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
             }
         };
 
-        int i = sub;
+        // this lane's host groups: sub, sub + L, ...; the opening has dealt with the slice's first ones
+        int g = sub;
+        if (t == tile_begin)
+            while (g < kOpeningHosts / 4) g += L;
         if constexpr (TWO_LEVELS) {
-            auto chunk1 = [&](auto width, int i0) {
+            // first level of W / 4 host groups (g0, g0 + L, ...) against the Q requests
+            auto chunk1 = [&](auto width, int g0) {
                 constexpr int W = decltype(width)::value;
                 unsigned int h1[W];
-                if constexpr (L == 1 && W >= 8) {
-                    // consecutive hosts: 128-bit shared-memory loads (i0 is a multiple of W)
 #pragma unroll
-                    for (int v = 0; v < W / 4; ++v) {
-                        const uint4 a = *reinterpret_cast<const uint4 *>(R1 + i0 + 4 * v);
-                        h1[4 * v] = a.x; h1[4 * v + 1] = a.y; h1[4 * v + 2] = a.z; h1[4 * v + 3] = a.w;
-                    }
-                } else {
-#pragma unroll
-                    for (int u = 0; u < W; ++u) h1[u] = R1[i0 + u * L];
+                for (int v = 0; v < W / 4; ++v) {
+                    const uint4 a = *reinterpret_cast<const uint4 *>(R1 + 4 * (g0 + v * L));
+                    h1[4 * v] = a.x; h1[4 * v + 1] = a.y; h1[4 * v + 2] = a.z; h1[4 * v + 3] = a.w;
                 }
                 unsigned int groups_passed = ranked_l1_chunk_groups_passed<Q, W>(r1, h1, guards1);
-                if (groups_passed) {
-                    if constexpr (W >= 8) {
-                        // second level only for the groups of four hosts in which a pair passed
-                        do {
-                            const int v = __ffs(groups_passed) - 1;
-                            groups_passed &= groups_passed - 1u;
-                            chunk2(std::integral_constant<int, 4>{}, i0 + 4 * v * L);
-                        } while (groups_passed);
-                    } else {
-                        chunk2(std::integral_constant<int, W>{}, i0);
-                    }
+                // second level only for the groups of four hosts in which a pair passed
+                while (groups_passed) {
+                    const int v = __ffs(groups_passed) - 1;
+                    groups_passed &= groups_passed - 1u;
+                    group2(g0 + v * L);
                 }
             };
-#ifndef NBOS_L1_WIDE
-#define NBOS_L1_WIDE 16   // hosts per first-level chunk of a lane
-#endif
-            for (; i + (NBOS_L1_WIDE - 1) * L < hosts; i += NBOS_L1_WIDE * L) chunk1(std::integral_constant<int, NBOS_L1_WIDE>{}, i);
-            for (; i + 3 * L < hosts; i += 4 * L) chunk1(std::integral_constant<int, 4>{}, i);
-            for (; i < hosts; i += L) chunk1(std::integral_constant<int, 1>{}, i);
+            for (; g + 3 * L < n_groups; g += 4 * L) chunk1(std::integral_constant<int, 16>{}, g);
+            for (; g < n_groups; g += L) chunk1(std::integral_constant<int, 4>{}, g);
         } else {
-            for (; i + 3 * L < hosts; i += 4 * L) chunk2(std::integral_constant<int, 4>{}, i);
-            for (; i < hosts; i += L) chunk2(std::integral_constant<int, 1>{}, i);
+            for (; g < n_groups; g += L) group2(g);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(empty_bar + 8u * s);
@@ -1055,6 +1107,7 @@ void fill_params(PlaceParams &p, const nbos_snapshot *s, const int32_t *d_reques
     p.total = (long long)s->N * batch;
     p.first_req = 0;
     p.n_req = p.total;
+    p.per_snapshot = 0;
     p.N = s->N;
     p.Hpad = s->Hpad;
     p.id_mask = (1u << s->key.bits_id) - 1u;
@@ -1067,11 +1120,12 @@ bool is_pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
 // shared memory, resident blocks per SM and lanes per request.
 struct LaunchPlan {
     int mode, T, tiles_total, per_sm, blocks_per_sm, L;
+    int per_snapshot;  // > 0: that many blocks per snapshot, no block works on two snapshots
     size_t smem;
 };
 
 int make_plan(const nbos_snapshot *s, long long total, long long batch, const nbos_launch_config &c,
-              LaunchPlan &plan)
+              bool whole_batch, LaunchPlan &plan)
 {
     const int mode = snapshot_mode(s, c.pair_mode);
     const int record = mode_record_bytes(mode);
@@ -1101,6 +1155,7 @@ int make_plan(const nbos_snapshot *s, long long total, long long batch, const nb
     // because each block then gets more requests and its last pass is fuller.
     int L = c.lanes_per_request;
     int blocks_per_sm = per_sm;
+    plan.per_snapshot = 0;
     {
         const bool two_level = mode == MODE_RANKED2;
         const double pair_cost = two_level ? 1.8 : (mode_is_sorted(mode) || mode_is_ranked(mode)) ? 3.0 : mode_is_grouped(mode) ? 3.3
@@ -1126,32 +1181,56 @@ int make_plan(const nbos_snapshot *s, long long total, long long batch, const nb
                 if (ctas > slots) ctas = slots;
                 long long n_req = (total + ctas - 1) / ctas;
                 n_req = (n_req + 31) / 32 * 32;
-                // the block's range is cut at snapshot boundaries, each piece into passes
-                double instr = 0.0;
-                const long long pieces = n_req > B ? n_req / B : 1;
-                const long long piece_len = n_req > B ? B : n_req, tail_len = n_req > B ? n_req % B : 0;
-                for (int part = 0; part < 2; ++part) {
-                    const long long len = part ? tail_len : piece_len, times = part ? 1 : pieces;
-                    if (len <= 0) continue;
+                auto pass = [&](int qq) {
+                    return kPassCost + qq * kRequestCost + per_host * (kHostCost + pair_cost * qq) + lg * qq * kMergeCost;
+                };
+                // instructions for `len` requests of one snapshot: full passes, then one that covers the rest
+                auto piece = [&](long long len) {
+                    if (len <= 0) return 0.0;
                     const long long full = len / (groups * max_q_kernel), rem = len % (groups * max_q_kernel);
                     int q = max_q_kernel;
                     while (q > 2 && (long long)(q >> 1) * groups >= rem) q >>= 1;
-                    auto pass = [&](int qq) {
-                        return kPassCost + qq * kRequestCost + per_host * (kHostCost + pair_cost * qq) + lg * qq * kMergeCost;
-                    };
-                    instr += (double)times * ((double)full * pass(max_q_kernel) + (rem ? pass(q) : 0.0));
-                    // a range that does not line up with the snapshots leaves some block a sliver of
-                    // another snapshot: one more pass over all hosts for a few requests
-                    if (part == 0 && total > B && (B % n_req != 0)) instr += pass(2);
+                    return (double)full * pass(max_q_kernel) + (rem ? pass(q) : 0.0);
+                };
+                // the block's range is cut at snapshot boundaries, each piece into passes
+                double instr = 0.0;
+                if (n_req > B) {
+                    instr = (double)(n_req / B) * piece(B) + piece(n_req % B);
+                    if (B % n_req != 0) instr += pass(2);
+                } else if (total > B && (B % n_req != 0)) {
+                    // ranges that do not line up with the snapshots: some block gets the end of one
+                    // snapshot and the start of the next, two partial pieces; the launch takes as long
+                    // as the unluckiest split
+                    for (int num = 1; num <= 4; ++num) {
+                        const long long a = (n_req * num / 5 + 31) / 32 * 32;
+                        const double two = piece(a) + piece(n_req - a);
+                        if (two > instr) instr = two;
+                    }
+                } else {
+                    instr = piece(n_req);
                 }
-                const long long on_sm = (ctas + s->sm_count - 1) / s->sm_count;
-                const int resident = (int)(on_sm < j ? on_sm : j);
-                const double cost = (double)on_sm * instr / issue_rate[resident > 4 ? 3 : resident - 1];
-                if (!have || cost < best * 0.99) {
-                    have = true;
-                    best = cost;
-                    L = cand;
-                    blocks_per_sm = j;
+                auto consider = [&](double instr_block, long long blocks, int per_snapshot) {
+                    const long long on_sm = (blocks + s->sm_count - 1) / s->sm_count;
+                    const int resident = (int)(on_sm < j ? on_sm : j);
+                    const double cost = (double)on_sm * instr_block / issue_rate[resident > 4 ? 3 : resident - 1];
+                    if (!have || cost < best * 0.99) {
+                        have = true;
+                        best = cost;
+                        L = cand;
+                        blocks_per_sm = j;
+                        plan.per_snapshot = per_snapshot;
+                    }
+                };
+                consider(instr, ctas, 0);
+                // several snapshots: also blocks that stay inside one snapshot, k per snapshot, all
+                // resident at once
+                if (whole_batch && total > B && !c.grid_blocks) {
+                    const long long n_snap = total / B;
+                    for (int k = 1; k <= 16 && n_snap * k <= slots; ++k) {
+                        const long long nb = (((B + 31) / 32 + k - 1) / k) * 32;
+                        if (nb < groups && k > 1) break;   // less than one request per group
+                        consider(piece(nb), n_snap * k, k);
+                    }
                 }
             }
         }
@@ -1212,7 +1291,8 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
     }
 
     LaunchPlan plan;
-    int rc = make_plan(s, total, batch, c, plan);
+    const bool whole_batch = range_first == 0 && total == (long long)s->N * batch;
+    int rc = make_plan(s, total, batch, c, whole_batch, plan);
     if (rc) return rc;
     const int mode = plan.mode, T = plan.T, tiles_total = plan.tiles_total;
     const int max_q_kernel = mode_max_q(mode);
@@ -1250,9 +1330,12 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
     if (cap < 1) cap = 1;
     if (c.grid_blocks) cap = c.grid_blocks;
     if (req_ctas > cap) req_ctas = cap;
+    const int per_snapshot = (K == 1 && !c.grid_blocks) ? plan.per_snapshot : 0;
+    if (per_snapshot > 0) req_ctas = (long long)s->N * per_snapshot;
 
     PlaceParams p;
     fill_params(p, s, d_requests, batch, d_out_hosts, d_out_found);
+    p.per_snapshot = per_snapshot;
     p.first_req = range_first;
     p.n_req = range_count;
     p.tile_hosts = T;
