@@ -54,6 +54,7 @@ def test_config2_full(nb):
     got, ref = both(nb, w)
     assert_same(got, ref, w.name)
     assert (ref[1] < 3).any() and (ref[1] == 3).any()  # sentinel path and full path both hit
+    check_properties(w, got[0], got[1])
 
 
 def test_config4_full(nb):
@@ -62,36 +63,57 @@ def test_config4_full(nb):
     assert_same(got, ref, w.name)
 
 
-def test_config3_full_size_sampled(nb):
-    """Full-size launch (4,096 hosts x 1,048,576 requests, the shape the benchmark times); the
-    checker recomputes a sample of the requests one by one; the rest is held to properties."""
+def test_config3_full(nb):
+    """Full-size launch (4,096 hosts x 1,048,576 requests, the shape the benchmark times), every
+    request compared with the checker (which runs on all host cores here), plus the properties
+    that hold at any size, checked without the checker."""
     w = W.make_config(3)
     hosts, found = nb.place_workload(w)
-    rng = np.random.default_rng(0)
-    ids = np.unique(np.concatenate([np.arange(0, 4096), np.arange(w.batch - 4096, w.batch),
-                                    rng.integers(0, w.batch, size=24576)]))
-    sub = dataclasses.replace(w, requests=np.ascontiguousarray(w.requests[:, ids]), batch=ids.size)
-    ref = oracle.place_workload(sub, threads=CPU_THREADS)
-    assert_same((hosts[:, ids], found[:, ids]), ref, "cfg3 sample")
-    # properties over the whole output
+    ref = oracle.place_workload(w, threads=CPU_THREADS)
+    assert_same((hosts, found), ref, "cfg3")
+    check_properties(w, hosts, found)
+
+
+def check_properties(w, hosts, found):
+    """Invariants of a placement, from the inputs alone: ids in range, -1 only at the tail, three
+    distinct hosts, every chosen host feasible, and no feasible host left out that ranks before
+    the worst chosen one (or at all, when fewer than three were found)."""
     assert hosts.min() >= -1 and hosts.max() < w.n_hosts
     filled = hosts >= 0
     np.testing.assert_array_equal(found, filled.sum(axis=-1))
     assert (filled[..., :-1] >= filled[..., 1:]).all()          # -1 only at the tail
-    h = hosts[0]
-    full = found[0] == 3
-    assert ((h[full, 0] != h[full, 1]) & (h[full, 1] != h[full, 2]) & (h[full, 0] != h[full, 2])).all()
-    # every chosen host passes the four capacity compares and the GPU test
-    req = w.requests[0]
-    for k in range(3):
-        sel = h[:, k] >= 0
-        hk = h[sel, k]
-        assert (req[sel, 0] <= w.gpus_total[0][hk]).all()
-        assert (req[sel, 1] <= w.vram_gb[0][hk]).all()
-        assert (req[sel, 2] <= w.millicpus[0][hk]).all()
-        assert (req[sel, 3] <= w.mem_mb[0][hk]).all()
-        assert ((w.gpus_subscribed[0][hk].astype(np.int64) + req[sel, 0]) * int(w.limit_den[0])
-                <= int(w.limit_num[0]) * w.gpus_total[0][hk].astype(np.int64) * 3).all()
+    rng = np.random.default_rng(5)
+    for n in range(w.n_snapshots):
+        h, req = hosts[n], w.requests[n].astype(np.int64)
+        full = found[n] == 3
+        assert ((h[full, 0] != h[full, 1]) & (h[full, 1] != h[full, 2]) & (h[full, 0] != h[full, 2])).all()
+        G, S, C = (getattr(w, k)[n].astype(np.int64) for k in ("gpus_total", "gpus_subscribed", "gpus_committed"))
+        num, den = int(w.limit_num[n]), int(w.limit_den[n])
+
+        def fits(r, hk):
+            return ((r[:, 0] <= G[hk]) & (r[:, 1] <= w.vram_gb[n][hk]) & (r[:, 2] <= w.millicpus[n][hk]) &
+                    (r[:, 3] <= w.mem_mb[n][hk]) & ((S[hk] + r[:, 0]) * den <= num * G[hk] * w.replicas_R) &
+                    (G[hk] >= 1) & (r.min(axis=1) >= 0))
+        for k in range(3):
+            sel = h[:, k] >= 0
+            assert fits(req[sel], h[sel, k]).all()
+        # a sample of requests against every host: nothing feasible ranks before the worst chosen
+        ids = rng.choice(w.batch, size=min(512, w.batch), replace=False)
+        for i in ids:
+            r = req[i:i + 1]
+            feas = fits(np.repeat(r, w.n_hosts, axis=0), np.arange(w.n_hosts))
+            assert int(feas.sum()) >= int(found[n, i]) and (found[n, i] == 3 or int(feas.sum()) == found[n, i])
+            if found[n, i] == 0:
+                continue
+            worst = h[i, found[n, i] - 1]
+            # order: idle GPUs descending, (S + g) / G ascending (exact, cross-multiplied), id ascending
+            idle = G - C
+            g = int(r[0, 0])
+            cand = np.nonzero(feas)[0]
+            better = (idle[cand] > idle[worst]) | ((idle[cand] == idle[worst]) & (
+                ((S[cand] + g) * G[worst] < (S[worst] + g) * G[cand]) |
+                (((S[cand] + g) * G[worst] == (S[worst] + g) * G[cand]) & (cand < worst))))
+            assert set(cand[better].tolist()) == set(h[i, :found[n, i] - 1].tolist())
 
 
 # ---- every launch shape gives the same bytes --------------------------------------------------
