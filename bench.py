@@ -654,7 +654,7 @@ def run_ours(args):
             nb.nbos_snapshot_destroy(sn)
 
     rot_mib = n_rot * w.n_snapshots * my_batch * 32 / 2**20
-    launches_per_step = 5  # scan, emit, rank, finalize (derivation, same kernels for create and refresh) + placement
+    launches_per_step = 3  # emit (+ validation), rank + finalize (snapshot refresh), placement
     line = {
         "metric": "placement decisions/sec", "value": value, "unit": "decisions/s",
         "pairs_per_s": value * w.n_hosts, "n_gpus": world, "steps": args.steps,

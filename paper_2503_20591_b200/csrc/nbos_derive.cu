@@ -21,13 +21,6 @@ struct ScanArgs {
     longlong2 limit0;         // used instead of limits[0] when `limits` is null (single snapshot)
     SnapStats *stats;
     int H, R, flags;
-    // update mode (null status = create mode): the new state must fit the layout chosen when the
-    // snapshot was created; a host that does not raises STATUS_STALE_LAYOUT in the status word
-    unsigned int *status;
-    const long long *lambda;   // per snapshot; null = static key
-    const int *g_single;       // per snapshot: the one GPU count of a static-key snapshot (0 = none)
-    unsigned long long sr_field_max;
-    int idle_max, pack_enabled, fmax[4];
 };
 
 // `num_r` is the limit's numerator times R (R already cancelled for the dynamic limit).
@@ -128,7 +121,6 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
     int idle_max = 0, g_min_inv = 0;  // INT_MAX - smallest G seen, 0 = none
     unsigned long long sub_max = 0ull;
     int max_gcap1 = 0, max_av = 0, max_ac = 0, max_am = 0;  // max_gcap1 = largest gmax + 1
-    unsigned int upd = 0u;
     for (int h = blockIdx.x * blockDim.x + threadIdx.x; h < a.H; h += gridDim.x * blockDim.x) {
         const size_t i = (size_t)n * a.H + h;
         const int G = a.G[i], S = a.S[i], C = a.C[i];
@@ -153,30 +145,6 @@ __global__ void __launch_bounds__(256) scan_kernel(const ScanArgs a)
         max_av = max(max_av, a.AV[i]);
         max_ac = max(max_ac, a.AC[i]);
         max_am = max(max_am, a.AM[i]);
-        if (a.status) {
-            bool stale = G - C > a.idle_max;
-            long long w = 1;
-            if (G >= 1) {
-                if (a.lambda) {
-                    const long long lam = a.lambda[n];
-                    if (lam % G) stale = true; else w = lam / G;
-                } else if (G != a.g_single[n]) {
-                    stale = true;
-                }
-            }
-            if (gm >= 0) {
-                unsigned long long top = (unsigned long long)S + (unsigned long long)gm;
-                if (a.flags & NBOS_ROOM_FOR_COMMITS) top = max(top, (unsigned long long)((lim.x * (long long)G) / lim.y));
-                if (top > a.sr_field_max / (unsigned long long)w) stale = true;
-            }
-            if (a.pack_enabled && (gm > a.fmax[0] || a.AV[i] > a.fmax[1] || a.AC[i] > a.fmax[2] || a.AM[i] > a.fmax[3]))
-                stale = true;
-            if (stale) upd |= STATUS_STALE_LAYOUT;
-        }
-    }
-    if (a.status) {
-        if (err) upd |= STATUS_BAD_VALUES;
-        if (upd) atomicOr(a.status, upd);
     }
     if (err) atomicOr(&s_err, err);
     atomicMax(&s_idle_max, idle_max);
@@ -215,6 +183,14 @@ struct EmitArgs {
     int idle_max;             // over all snapshots: the idle field stores idle_max - (G - C)
     int bits_idle, bits_sr, bits_id;
     int group_major;          // 1: visiting order is (GPU count, key at g = 0) instead of the key alone
+    unsigned int *done;       // [N][ceil(Hpad / 256)] counters of rank_kernel, cleared here (null = unused)
+    // update mode (null status = create mode, where scan_kernel has validated the state): the new
+    // state must be valid and fit the layout chosen when the snapshot was created; a host that is
+    // not or does not raises the status word instead
+    unsigned int *status;
+    const int *g_single;       // per snapshot: the one GPU count of a static-key snapshot (0 = none)
+    unsigned long long sr_field_max;
+    int check_fmax, fmax[4];
 };
 
 constexpr int kMaxGpuCountGroups = 8;  // distinct GPU counts per snapshot up to which the table is grouped
@@ -228,6 +204,7 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
     const int n = blockIdx.y;
     const int h = blockIdx.x * blockDim.x + threadIdx.x;
     if (h >= a.Hpad) return;
+    if (a.done && h < (a.Hpad + 255) / 256) a.done[(size_t)n * ((a.Hpad + 255) / 256) + h] = 0u;
     int4 f = make_int4(-1, 0, 0, 0);  // padding host: takes nothing
     int4 sq = make_int4(-1, -1, 0, 0);
     KeyT A = (KeyT)h, B = 0;
@@ -236,7 +213,38 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
         const size_t i = (size_t)n * a.H + h;
         const int G = a.G[i], S = a.S[i], C = a.C[i];
         const longlong2 lim = a.limits ? a.limits[n] : a.limit0;
-        const int gm = derive_gmax(G, S, C, lim.x, lim.y, a.flags);
+        int gm = derive_gmax(G, S, C, lim.x, lim.y, a.flags);
+        if (a.status) {
+            // the checks scan_kernel makes at creation, against the stored layout
+            unsigned int upd = 0u;
+            if ((G | S | C | a.AV[i] | a.AC[i] | a.AM[i]) < 0 || C > G || G > NBOS_MAX_GPUS_PER_HOST) {
+                upd = STATUS_BAD_VALUES;
+                gm = -1;   // the tables are undefined after such an update; keep the arithmetic in range
+            } else {
+                bool stale = G - C > a.idle_max;
+                long long w = 1;
+                if (G >= 1) {
+                    if (a.lambda) {
+                        const long long lam = a.lambda[n];
+                        if (lam % G) stale = true; else w = lam / G;
+                    } else if (G != a.g_single[n]) {
+                        stale = true;
+                    }
+                }
+                if (gm >= 0) {
+                    unsigned long long top = (unsigned long long)S + (unsigned long long)gm;
+                    if (a.flags & NBOS_ROOM_FOR_COMMITS) top = max(top, (unsigned long long)((lim.x * (long long)G) / lim.y));
+                    if (top > a.sr_field_max / (unsigned long long)w) stale = true;
+                }
+                if (a.check_fmax && (gm > a.fmax[0] || a.AV[i] > a.fmax[1] || a.AC[i] > a.fmax[2] || a.AM[i] > a.fmax[3]))
+                    stale = true;
+                if (stale) {
+                    upd = STATUS_STALE_LAYOUT;
+                    gm = -1;
+                }
+            }
+            if (upd) atomicOr(a.status, upd);
+        }
         f = make_int4(gm, a.AV[i], a.AC[i], a.AM[i]);
         sq.z = S;
         if (G >= 1 && lim.y >= 1) {
@@ -271,29 +279,6 @@ __global__ void __launch_bounds__(256) emit_kernel(const EmitArgs a)
     reinterpret_cast<PairT *>(a.ab)[(size_t)n * a.Hpad + h] = p;
 }
 
-// Visiting order: hosts are visited in ascending order of their key at g = 0 (hosts that take
-// nothing last), which makes later hosts rarely displace an earlier best-three entry. The sort
-// keys are unique, so the position of host i is the number of hosts with a smaller key. Each
-// block counts, for 256 hosts, the smaller keys inside one chunk of kRankChunk keys staged in
-// shared memory, and adds its partial count to rank[i]. grid (ceil(Hpad/256), ceil(Hpad/chunk), N).
-constexpr int kRankChunk = 256;
-__global__ void __launch_bounds__(256) rank_kernel(const unsigned long long *sortkey, unsigned int *rank, int Hpad)
-{
-    __shared__ unsigned long long chunk[kRankChunk];
-    const size_t base = (size_t)blockIdx.z * Hpad;
-    const int j0 = blockIdx.y * kRankChunk;
-    const int nj = min(kRankChunk, Hpad - j0);
-    for (int j = threadIdx.x; j < nj; j += blockDim.x) chunk[j] = sortkey[base + j0 + j];
-    __syncthreads();
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= Hpad) return;
-    const unsigned long long ki = sortkey[base + i];
-    unsigned int smaller = 0;
-#pragma unroll 8
-    for (int j = 0; j < nj; ++j) smaller += chunk[j] < ki ? 1u : 0u;
-    if (smaller) atomicAdd(&rank[base + i], smaller);
-}
-
 struct FinalizeArgs {
     const int4 *tmp_feas;
     const void *tmp_ab;
@@ -308,13 +293,12 @@ struct FinalizeArgs {
     RankLayout ranked;
 };
 
-// grid (ceil(Hpad / 256), N): move the records into visiting order and build the packed form.
+// Move the record of host `src` of snapshot `n` to its place in visiting order and build the
+// packed and ranked forms there.
 template <typename PairT>
-__global__ void __launch_bounds__(256) finalize_kernel(const FinalizeArgs a)
+__device__ __forceinline__ void finalize_host(const FinalizeArgs &a, int n, int src)
 {
-    const int src = blockIdx.x * blockDim.x + threadIdx.x;
-    if (src >= a.Hpad) return;
-    const size_t base = (size_t)blockIdx.y * a.Hpad;
+    const size_t base = (size_t)n * a.Hpad;
     const unsigned int j = a.rank ? a.rank[base + src] : (unsigned int)src;
     const int4 f = a.tmp_feas[base + src];
     const PairT p = reinterpret_cast<const PairT *>(a.tmp_ab)[base + src];
@@ -345,6 +329,54 @@ __global__ void __launch_bounds__(256) finalize_kernel(const FinalizeArgs a)
             a.rk1[base + j] = w1;
         }
     }
+}
+
+// grid (ceil(Hpad / 256), N): tables that keep host order (too large to rank).
+template <typename PairT>
+__global__ void __launch_bounds__(256) finalize_kernel(const FinalizeArgs a)
+{
+    const int src = blockIdx.x * blockDim.x + threadIdx.x;
+    if (src < a.Hpad) finalize_host<PairT>(a, blockIdx.y, src);
+}
+
+// Visiting order: hosts are visited in ascending order of their key at g = 0 (hosts that take
+// nothing last), which makes later hosts rarely displace an earlier best-three entry. The sort
+// keys are unique, so the position of host i is the number of hosts with a smaller key. Each
+// block counts, for 256 hosts, the smaller keys inside one chunk of kRankChunk keys staged in
+// shared memory, and adds its partial count to rank[i]; the block that is the last of its 256
+// hosts' blocks to finish (a counter per group of 256 hosts tells) finds their positions
+// complete and moves their records into place (finalize_host) in the same launch.
+// grid (ceil(Hpad/256), ceil(Hpad/chunk), N); rank[] and done[] must be zero.
+constexpr int kRankChunk = 256;
+template <typename PairT>
+__global__ void __launch_bounds__(256) rank_finalize_kernel(const unsigned long long *sortkey, unsigned int *rank,
+                                                            unsigned int *done, const FinalizeArgs fa)
+{
+    __shared__ unsigned long long chunk[kRankChunk];
+    __shared__ unsigned int s_last;
+    const int Hpad = fa.Hpad;
+    const size_t base = (size_t)blockIdx.z * Hpad;
+    const int j0 = blockIdx.y * kRankChunk;
+    const int nj = min(kRankChunk, Hpad - j0);
+    for (int j = threadIdx.x; j < nj; j += blockDim.x) chunk[j] = sortkey[base + j0 + j];
+    __syncthreads();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < Hpad) {
+        const unsigned long long ki = sortkey[base + i];
+        unsigned int smaller = 0;
+#pragma unroll 8
+        for (int j = 0; j < nj; ++j) smaller += chunk[j] < ki ? 1u : 0u;
+        if (smaller) atomicAdd(&rank[base + i], smaller);
+    }
+    // every thread's additions are visible device-wide before the block signs off
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0)
+        s_last = atomicAdd(&done[(size_t)blockIdx.z * gridDim.x + blockIdx.x], 1u) == gridDim.y - 1 ? 1u : 0u;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();   // the other blocks' additions, published before their sign-off, are read below
+    if (i < Hpad) finalize_host<PairT>(fa, blockIdx.z, i);
 }
 
 int bits_for(unsigned long long max_value)
@@ -390,6 +422,7 @@ Layout workspace_layout(int N, int Hpad)
     l.off_tmp_seq = o; o = up(o + (size_t)N * Hpad * sizeof(int4));
     l.off_sortkey = o; o = up(o + (size_t)N * Hpad * sizeof(unsigned long long));
     l.off_perm = o;    o = up(o + (size_t)N * Hpad * sizeof(unsigned int));
+    l.off_done = o;    o = up(o + (size_t)N * ((Hpad + 255) / 256) * sizeof(unsigned int));
     l.total = o;
     return l;
 }
@@ -457,8 +490,9 @@ int stage_limits(DeriveCtx &c, const nbos_snapshot_desc *d, bool first_time)
     return NBOS_OK;
 }
 
-// emit -> rank -> finalize with the layout stored in the handle
-int emit_tables(DeriveCtx &c)
+// emit -> rank + finalize with the layout stored in the handle. `check_state` (refresh of an
+// existing snapshot): the emit kernel also validates the new state against that layout.
+int emit_tables(DeriveCtx &c, bool check_state)
 {
     nbos_snapshot *s = c.s;
     const int N = s->N, H = s->H, Hpad = s->Hpad;
@@ -469,25 +503,36 @@ int emit_tables(DeriveCtx &c)
     unsigned long long *sortkey = reinterpret_cast<unsigned long long *>(c.ws + c.lay.off_sortkey);
     unsigned int *perm = reinterpret_cast<unsigned int *>(c.ws + c.lay.off_perm);
     int4 *tmp_seq = reinterpret_cast<int4 *>(c.ws + c.lay.off_tmp_seq);
+    unsigned int *done = reinterpret_cast<unsigned int *>(c.ws + c.lay.off_done);
+    const int *fm = s->pack.enabled ? s->pack.fmax : s->rank.fmax;  // the same values in both layouts
     EmitArgs ea{c.G, c.S, c.C, c.AV, c.AC, c.AM, c.limits_arg, c.limit0, k.static_key ? nullptr : d_lambda,
                 s->presorted ? perm : nullptr, tmp_feas, tmp_seq, tmp_ab, sortkey,
                 H, Hpad, s->R, s->flags, s->key_order, s->idle_max, k.bits_idle, k.bits_sr, k.bits_id,
-                k.grouped};
+                k.grouped, s->presorted ? done : nullptr,
+                check_state ? s->d_update_status : nullptr,
+                reinterpret_cast<const int *>(c.ws + c.lay.off_g_single),
+                k.bits_sr >= 64 ? ~0ull : ((1ull << k.bits_sr) - 1ull),
+                (s->pack.enabled || s->rank.enabled) ? 1 : 0, {fm[0], fm[1], fm[2], fm[3]}};
     dim3 grid((Hpad + 255) / 256, N);
     if (k.key_bits == 32)
         emit_kernel<unsigned int, uint2><<<grid, 256, 0, c.stream>>>(ea);
     else
         emit_kernel<unsigned long long, ulonglong2><<<grid, 256, 0, c.stream>>>(ea);
-    if (s->presorted)
-        rank_kernel<<<dim3((Hpad + 255) / 256, (Hpad + kRankChunk - 1) / kRankChunk, N), 256, 0, c.stream>>>(sortkey, perm, Hpad);
     FinalizeArgs fa{tmp_feas, tmp_ab, s->presorted ? perm : nullptr, reinterpret_cast<int4 *>(c.ws + c.lay.off_feas),
                     c.ws + c.lay.off_ab, reinterpret_cast<uint4 *>(c.ws + c.lay.off_pk),
                     reinterpret_cast<uint2 *>(c.ws + c.lay.off_rk),
                     reinterpret_cast<unsigned int *>(c.ws + c.lay.off_rk1), Hpad, s->pack, s->rank};
-    if (k.key_bits == 32)
+    if (s->presorted) {
+        const dim3 rgrid((Hpad + 255) / 256, (Hpad + kRankChunk - 1) / kRankChunk, N);
+        if (k.key_bits == 32)
+            rank_finalize_kernel<uint2><<<rgrid, 256, 0, c.stream>>>(sortkey, perm, done, fa);
+        else
+            rank_finalize_kernel<ulonglong2><<<rgrid, 256, 0, c.stream>>>(sortkey, perm, done, fa);
+    } else if (k.key_bits == 32) {
         finalize_kernel<uint2><<<grid, 256, 0, c.stream>>>(fa);
-    else
+    } else {
         finalize_kernel<ulonglong2><<<grid, 256, 0, c.stream>>>(fa);
+    }
     NBOS_CUDA_TRY(cudaGetLastError());
     return NBOS_OK;
 }
@@ -532,8 +577,7 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
 
     int rc = stage_limits(c, d, true);
     if (rc) return rc;
-    ScanArgs sa{d_G, d_S, d_C, d_AV, d_AC, d_AM, c.limits_arg, c.limit0, d_stats, H, s->R, s->flags,
-                nullptr, nullptr, nullptr, 0ull, 0, 0, {0, 0, 0, 0}};
+    ScanArgs sa{d_G, d_S, d_C, d_AV, d_AC, d_AM, c.limits_arg, c.limit0, d_stats, H, s->R, s->flags};
     scan_kernel<<<dim3(c.bx, N), 256, 0, stream>>>(sa);
     NBOS_CUDA_TRY(cudaGetLastError());
     NBOS_CUDA_TRY(cudaMemcpyAsync(h_stats, d_stats, sizeof(SnapStats) * (size_t)N,
@@ -725,7 +769,7 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
         NBOS_CUDA_TRY(cudaMemcpyAsync(d_lambda, h_lambda, sizeof(long long) * (size_t)N, cudaMemcpyHostToDevice, stream));
     NBOS_CUDA_TRY(cudaMemcpyAsync(d_g_single, h_g_single, sizeof(int) * (size_t)N, cudaMemcpyHostToDevice, stream));
 
-    rc = emit_tables(c);
+    rc = emit_tables(c, false);
     if (rc) return rc;
     s->d_status = reinterpret_cast<unsigned int *>(c.ws + c.lay.off_status);
     s->d_update_status = reinterpret_cast<unsigned int *>(c.ws + c.lay.off_status + kUpdateStatusOffset);
@@ -741,8 +785,9 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
 }
 
 // Re-derive the tables of an existing snapshot from new state, keeping the key and packing layout
-// chosen at creation. Nothing is read back: a state that does not fit the layout is reported
-// through the status word.
+// chosen at creation: two kernels (emit, which also validates the state against that layout, and
+// rank + finalize). Nothing is read back: a state that is invalid or does not fit the layout is
+// reported through the status word.
 int update_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t *d_G,
                     const int32_t *d_S, const int32_t *d_C, const int32_t *d_AV,
                     const int32_t *d_AC, const int32_t *d_AM, cudaStream_t stream)
@@ -750,18 +795,7 @@ int update_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     DeriveCtx c = make_ctx(s, d_G, d_S, d_C, d_AV, d_AC, d_AM, stream);
     int rc = stage_limits(c, d, false);
     if (rc) return rc;
-    const int *fm = s->pack.enabled ? s->pack.fmax : s->rank.fmax;  // the same values in both layouts
-    ScanArgs sa{d_G, d_S, d_C, d_AV, d_AC, d_AM, c.limits_arg, c.limit0,
-                reinterpret_cast<SnapStats *>(c.ws + c.lay.off_stats), s->H, s->R, s->flags,
-                s->d_update_status,
-                s->key.static_key ? nullptr : reinterpret_cast<const long long *>(c.ws + c.lay.off_lambda),
-                reinterpret_cast<const int *>(c.ws + c.lay.off_g_single),
-                s->key.bits_sr >= 64 ? ~0ull : ((1ull << s->key.bits_sr) - 1ull), s->idle_max,
-                s->pack.enabled || s->rank.enabled,
-                {fm[0], fm[1], fm[2], fm[3]}};
-    scan_kernel<<<dim3(c.bx, s->N), 256, 0, stream>>>(sa);
-    NBOS_CUDA_TRY(cudaGetLastError());
-    return emit_tables(c);
+    return emit_tables(c, true);
 }
 
 }  // namespace nbos

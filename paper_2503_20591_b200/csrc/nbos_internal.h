@@ -47,7 +47,7 @@ enum : unsigned int {
 
 struct Layout {
     size_t off_status, off_limits, off_sums, off_stats, off_lambda, off_g_single, off_feas, off_ab, off_pk, off_rk, off_rk1;
-    size_t off_tmp_feas, off_tmp_ab, off_tmp_seq, off_sortkey, off_perm, total;
+    size_t off_tmp_feas, off_tmp_ab, off_tmp_seq, off_sortkey, off_perm, off_done, total;
 };
 Layout workspace_layout(int n_snapshots, int hosts_padded);
 inline int pad_hosts(int h) { return (h + 31) & ~31; }
