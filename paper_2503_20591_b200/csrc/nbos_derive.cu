@@ -193,7 +193,7 @@ struct EmitArgs {
     int check_fmax, fmax[4];
 };
 
-constexpr int kMaxGpuCountGroups = 8;  // distinct GPU counts per snapshot up to which the table is grouped
+constexpr int kMaxGpuCountGroups = kGroupSlices;  // distinct GPU counts per snapshot up to which the table is grouped
 constexpr int kSortMaxHosts = 65536;  // larger tables keep host order (ranking is quadratic in the host count)
 constexpr unsigned long long kSortNever = 0xFFFFFFFF00000000ull;  // hosts that take nothing go last (| host index)
 
@@ -379,6 +379,44 @@ __global__ void __launch_bounds__(256) rank_finalize_kernel(const unsigned long 
     if (i < Hpad) finalize_host<PairT>(fa, blockIdx.z, i);
 }
 
+// Grouped tables (hosts stored GPU count by GPU count): where each group starts. A position
+// starts a group when its key slope differs from its predecessor's; the hosts that take nothing
+// are stored last and end the last group. One block per snapshot; bounds[n][k] = start of group k
+// for k < number of groups, = end of the last group after that.
+__global__ void __launch_bounds__(256) group_bounds_kernel(const int4 *feas, const uint2 *ab, int Hpad, int *bounds)
+{
+    __shared__ int s_start[kGroupSlices + 1];
+    __shared__ int s_count, s_end;
+    const size_t base = (size_t)blockIdx.x * Hpad;
+    if (threadIdx.x == 0) {
+        s_count = 0;
+        s_end = Hpad;
+    }
+    __syncthreads();
+    for (int pos = threadIdx.x; pos < Hpad; pos += blockDim.x) {
+        const bool live = feas[base + pos].x >= 0;
+        const bool prev_live = pos > 0 && feas[base + pos - 1].x >= 0;
+        if (!live) {
+            if (pos == 0 || prev_live) atomicMin(&s_end, pos);
+        } else if (pos == 0 || ab[base + pos].y != ab[base + pos - 1].y) {
+            const int slot = atomicAdd(&s_count, 1);
+            if (slot <= kGroupSlices) s_start[slot] = pos;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int n = s_count < kGroupSlices ? s_count : kGroupSlices;
+        for (int i = 1; i < n; ++i) {       // a handful of entries: insertion sort
+            const int v = s_start[i];
+            int j = i - 1;
+            for (; j >= 0 && s_start[j] > v; --j) s_start[j + 1] = s_start[j];
+            s_start[j + 1] = v;
+        }
+        int *out = bounds + (size_t)blockIdx.x * (kGroupSlices + 1);
+        for (int k = 0; k <= kGroupSlices; ++k) out[k] = k < n ? s_start[k] : s_end;
+    }
+}
+
 int bits_for(unsigned long long max_value)
 {
     int b = 0;
@@ -423,6 +461,7 @@ Layout workspace_layout(int N, int Hpad)
     l.off_sortkey = o; o = up(o + (size_t)N * Hpad * sizeof(unsigned long long));
     l.off_perm = o;    o = up(o + (size_t)N * Hpad * sizeof(unsigned int));
     l.off_done = o;    o = up(o + (size_t)N * ((Hpad + 255) / 256) * sizeof(unsigned int));
+    l.off_gbounds = o; o = up(o + (size_t)N * (kGroupSlices + 1) * sizeof(int));
     l.total = o;
     return l;
 }
@@ -533,6 +572,9 @@ int emit_tables(DeriveCtx &c, bool check_state)
     } else {
         finalize_kernel<ulonglong2><<<grid, 256, 0, c.stream>>>(fa);
     }
+    if (k.grouped)
+        group_bounds_kernel<<<N, 256, 0, c.stream>>>(fa.feas, reinterpret_cast<const uint2 *>(fa.ab), Hpad,
+                                                     reinterpret_cast<int *>(c.ws + c.lay.off_gbounds));
     NBOS_CUDA_TRY(cudaGetLastError());
     return NBOS_OK;
 }
@@ -677,6 +719,12 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     }
     s->pack = pk;
     s->presorted = Hpad <= kSortMaxHosts;
+    // Hosts with different GPU counts rank differently for different asks, but within one GPU
+    // count the order is the same for every ask. With few distinct counts the table is stored
+    // count by count, each group in key order, and the placement kernel treats every group like
+    // a table in key order.
+    s->key.grouped = (!k.static_key && k.key_bits == 32 && pk.enabled && s->presorted &&
+                      max_distinct_g <= kMaxGpuCountGroups) ? 1 : 0;
 
     // Ranked form (see RankLayout): six slots -- three per word at the same bit positions -- for
     // the four capacities, the rank and one unused slot. Components are paired by width (the two
@@ -684,7 +732,7 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     // while the three widths exceed the 29 bits left beside the guards the widest slot that may
     // shrink does: the GPU component and the rank stay exact, the others lose low bits.
     RankLayout rl = {};
-    if (k.key_bits == 32 && k.static_key && s->presorted) {
+    if (k.key_bits == 32 && (k.static_key || s->key.grouped) && s->presorted) {
         int w6[6] = {width[0], width[1], width[2], width[3], bits_for((unsigned long long)(Hpad - 1)), 0};
         int order[6] = {0, 1, 2, 3, 4, 5};
         for (int i = 0; i < 6; ++i)
@@ -757,13 +805,6 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
         }
     }
     s->rank = rl;
-    // Hosts with different GPU counts rank differently for different asks, but within one GPU
-    // count the order is the same for every ask. With few distinct counts the table is stored
-    // count by count, each group in key order, and the placement kernel treats every group like
-    // a table in key order.
-    s->key.grouped = (!k.static_key && k.key_bits == 32 && pk.enabled && s->presorted &&
-                      max_distinct_g <= kMaxGpuCountGroups) ? 1 : 0;
-
     // what a later nbos_snapshot_update checks the new state against
     if (!k.static_key)
         NBOS_CUDA_TRY(cudaMemcpyAsync(d_lambda, h_lambda, sizeof(long long) * (size_t)N, cudaMemcpyHostToDevice, stream));
@@ -778,6 +819,7 @@ int derive_snapshot(nbos_snapshot *s, const nbos_snapshot_desc *d, const int32_t
     s->d_pk = reinterpret_cast<const uint4 *>(c.ws + c.lay.off_pk);
     s->d_rk = reinterpret_cast<const uint2 *>(c.ws + c.lay.off_rk);
     s->d_rk1 = reinterpret_cast<const unsigned int *>(c.ws + c.lay.off_rk1);
+    s->d_group_bounds = reinterpret_cast<const int *>(c.ws + c.lay.off_gbounds);
     s->d_host_feas = reinterpret_cast<const int4 *>(c.ws + c.lay.off_tmp_feas);
     s->d_host_ab = c.ws + c.lay.off_tmp_ab;
     s->d_host_seq = reinterpret_cast<const int4 *>(c.ws + c.lay.off_tmp_seq);

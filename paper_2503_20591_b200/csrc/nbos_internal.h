@@ -47,10 +47,12 @@ enum : unsigned int {
 
 struct Layout {
     size_t off_status, off_limits, off_sums, off_stats, off_lambda, off_g_single, off_feas, off_ab, off_pk, off_rk, off_rk1;
-    size_t off_tmp_feas, off_tmp_ab, off_tmp_seq, off_sortkey, off_perm, off_done, total;
+    size_t off_tmp_feas, off_tmp_ab, off_tmp_seq, off_sortkey, off_perm, off_done, off_gbounds, total;
 };
 Layout workspace_layout(int n_snapshots, int hosts_padded);
 inline int pad_hosts(int h) { return (h + 31) & ~31; }
+
+constexpr int kGroupSlices = 8;   // distinct GPU counts per snapshot up to which a table is stored count by count
 
 struct KeyLayout {
     int key_bits;  // 32 or 64
@@ -123,6 +125,10 @@ struct nbos_snapshot {
     nbos::PackLayout pack;
     const uint2 *d_rk;    // [N][Hpad] (word0, word1) of the ranked form, only when rank.enabled
     const unsigned int *d_rk1;  // [N][Hpad] first-level word of the ranked form, only when rank.l1_enabled
+    // [N][kGroupSlices + 1] table positions at which the GPU-count groups of a grouped snapshot
+    // start (entry k = start of group k; the entries after the last group = where the hosts that
+    // can take something end), only when key.grouped
+    const int *d_group_bounds;
     nbos::RankLayout rank;
     int presorted;
     int idle_max;             // the key's idle field stores idle_max - (G - C)

@@ -60,9 +60,14 @@ enum : int {
     MODE_RANKED2 = 11,       // as 10 behind a first level: one 32-bit word per host and per request, one
                              // subtraction + one logic operation per pair; chunks in which a pair passes
                              // go through the two-word test               (records: rk + rk1, then feas + ab)
-    MODE_COUNT = 12,
+    MODE_RANKED_GROUPS = 12,   // as 10 for a table stored GPU count by GPU count: a block walks the groups one
+                               // after the other, each like a table in key order; best three kept as keys
+    MODE_RANKED2_GROUPS = 13,  // as 11, likewise
+    MODE_COUNT = 14,
 };
-__host__ __device__ constexpr bool mode_is_ranked(int mode) { return mode == MODE_RANKED || mode == MODE_RANKED2; }
+__host__ __device__ constexpr bool mode_is_ranked(int mode) { return mode >= MODE_RANKED && mode <= MODE_RANKED2_GROUPS; }
+__host__ __device__ constexpr bool mode_ranked_two_levels(int mode) { return mode == MODE_RANKED2 || mode == MODE_RANKED2_GROUPS; }
+__host__ __device__ constexpr bool mode_ranked_by_group(int mode) { return mode == MODE_RANKED_GROUPS || mode == MODE_RANKED2_GROUPS; }
 __host__ __device__ constexpr bool mode_is_packed(int mode) { return mode >= MODE_PACKED && mode <= MODE_GROUPED2; }
 __host__ __device__ constexpr bool mode_is_sorted(int mode) { return mode == MODE_SORTED || mode == MODE_SORTED2; }
 __host__ __device__ constexpr bool mode_is_grouped(int mode) { return mode == MODE_GROUPED || mode == MODE_GROUPED2; }
@@ -70,7 +75,7 @@ __host__ __device__ constexpr bool mode_is_grouped(int mode) { return mode == MO
 __host__ __device__ constexpr bool mode_is_chained(int mode) { return mode_is_sorted(mode) || mode_is_grouped(mode); }
 __host__ __device__ constexpr bool mode_is_static(int mode) { return mode == MODE_PACKED_STATIC || mode == MODE_PACKED2_STATIC || mode_is_sorted(mode); }
 __host__ __device__ constexpr bool mode_two_masks(int mode) { return mode == MODE_PACKED2 || mode == MODE_PACKED2_STATIC || mode == MODE_SORTED2 || mode == MODE_GROUPED2; }
-__host__ __device__ constexpr int mode_record_bytes(int mode) { return mode == MODE_KEY64 ? 32 : mode == MODE_PLAIN ? 24 : mode == MODE_RANKED ? 8 : mode == MODE_RANKED2 ? 12 : 16; }
+__host__ __device__ constexpr int mode_record_bytes(int mode) { return mode == MODE_KEY64 ? 32 : mode == MODE_PLAIN ? 24 : mode_is_ranked(mode) ? (mode_ranked_two_levels(mode) ? 12 : 8) : 16; }
 __host__ __device__ constexpr int mode_max_q(int mode) { return mode == MODE_KEY64 ? 4 : 8; }
 // Resident blocks per SM the kernels are compiled for. The modes that rank hosts by their own key
 // touch most best-three registers only on the rare update path, so 64 registers (a few spills
@@ -97,6 +102,8 @@ struct PlaceParams {
     int N, Hpad;
     int tile_hosts, tiles_total, K, req_ctas;
     int per_snapshot;       // > 0: blocks do not share snapshots, each snapshot's requests go to this many blocks
+    const int *group_bounds;  // non-null: the K host slices are the GPU-count groups of each snapshot,
+                              // [N][kGroupSlices + 1] table positions (ranked form of grouped tables)
     unsigned int id_mask;
     int max_q;
 };
@@ -162,6 +169,38 @@ __device__ __forceinline__ void block_request_range(const PlaceParams &p, int cr
     if (hi > p.n_req) hi = p.n_req;
     lo += p.first_req;
     hi += p.first_req;
+}
+
+// ---- the host slice of a block -----------------------------------------------------------------
+// Hosts [lo, hi) of the table are staged (tile by tile), of which [real_lo, real_hi) are the
+// block's to evaluate. Ordinary slices are runs of whole tiles and the two ranges coincide. The
+// slices of a grouped table are its GPU-count groups, which start anywhere: the staged range is
+// widened to multiples of four hosts (16-byte copies), and what lies outside the group is ignored.
+struct SliceRange {
+    int lo, hi, real_lo, real_hi;
+};
+__device__ __forceinline__ SliceRange slice_range(const PlaceParams &p, int n, int slice)
+{
+    SliceRange r;
+    if (p.group_bounds) {
+        const int *b = p.group_bounds + (size_t)n * (kGroupSlices + 1);
+        r.real_lo = b[slice];
+        r.real_hi = b[slice + 1];
+        if (r.real_hi <= r.real_lo) {
+            r.lo = r.hi = r.real_lo = r.real_hi = 0;
+        } else {
+            r.lo = r.real_lo & ~3;
+            r.hi = (r.real_hi + 3) & ~3;
+        }
+    } else {
+        const int T = p.tile_hosts;
+        r.lo = (p.tiles_total * slice / p.K) * T;          // tiles_total * K stays far below 2^31
+        r.hi = (p.tiles_total * (slice + 1) / p.K) * T;
+        if (r.hi > p.Hpad) r.hi = p.Hpad;
+        r.real_lo = r.lo;
+        r.real_hi = r.hi;
+    }
+    return r;
 }
 
 // ---- the pair step --------------------------------------------------------------------------
@@ -489,34 +528,39 @@ __device__ __forceinline__ bool run_pass(const PlaceParams &p, unsigned char *st
 }
 
 // ---- one pass in ranked form ------------------------------------------------------------------
-// Same contract as run_pass. The best three of a request are kept as positions in the table
-// (which is stored in key order, so a smaller position is a smaller key) and turned into keys
-// after the last tile.
+// Same contract as run_pass. Inside one host slice (a run of tiles of a table in key order, or
+// one GPU-count group of a grouped table) a smaller position is a smaller key, so "would this
+// host enter the best three" is a compare of positions, which the packed words carry. A block
+// walks its slices [slice_first, slice_last) one after the other. With a single slice the best
+// three of a request are kept as positions (turned into keys after the last tile) and double as
+// the rank threshold; a block that walks the groups of a grouped table keeps them as keys across
+// the groups, and per group the positions of the first three hosts that fit give the threshold.
 //
 // Hosts are dealt to the L lanes of a request group in groups of four consecutive hosts (lane s
 // takes groups s, s + L, ...), so that a lane's host words come in 128-bit shared-memory loads
 // whatever L is.
 //
-// Opening. The first 16 hosts of the block's slice of the table are compared exactly (four
-// compares on the exact records) against every request of the pass, in table order, until a
-// request has three hosts: in a table in key order most requests find their three right there,
-// and the pair loop then starts with the rank thresholds already in the request words instead
-// of going through the second level and the exact test for its first chunks. Every lane of a
-// group does this (they all need the thresholds); lane 0 of the group keeps the finds.
+// Opening. The first 16 hosts of a slice are compared exactly (four compares on the exact
+// records) against every request of the pass, in table order, until a request has three hosts:
+// in a table in key order most requests find their three right there, and the pair loop then
+// starts with the rank thresholds already in the request words instead of going through the
+// second level and the exact test for its first chunks. Every lane of a group does this (they all
+// need the thresholds); lane 0 of the group keeps the finds.
 //
-// Pair loop, from host 16 on. Per pair: one subtraction and one logic operation on the
-// first-level words (TWO_LEVELS), or directly the two-word test. A group of four hosts in which
-// some pair passed the first level goes through the two-word test; pairs that pass that one too
-// are re-tested with the exact records, fitting hosts enter the best three, and the request's
-// rank fields are set from its new third best (or from the opening's, whichever is earlier).
+// Pair loop, from the end of the opening on. Per pair: one subtraction and one logic operation
+// on the first-level words (TWO_LEVELS), or directly the two-word test. A group of four hosts in
+// which some pair passed the first level goes through the two-word test; pairs that pass that
+// one too are re-tested with the exact records, fitting hosts enter the best three, and the
+// request's rank fields are set from the slice's new third fit (or from the opening's,
+// whichever is earlier).
 constexpr int kOpeningHosts = 16;
 
-template <int Q, int L, bool TWO_LEVELS>
+template <int Q, int L, bool TWO_LEVELS, bool BY_GROUP>
 __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned char *stages,
                                                 uint32_t stage_bytes, uint32_t full_bar,
                                                 uint32_t empty_bar, volatile unsigned int *abort_flag,
-                                                uint32_t &ring_pos, int tile_begin, int tile_end,
-                                                int slice, long long first, int count, int n)
+                                                uint32_t &ring_pos, int slice_first, int slice_last,
+                                                const SliceRange &own_slice, long long first, int count, int n)
 {
     constexpr unsigned int kNone = 0xFFFFFFFFu;
     constexpr int kGroups = kComputeThreads / L;
@@ -539,173 +583,232 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
         if ((r.x | r.y | r.z | r.w) < 0) r.x = INT_MAX;
         return r;
     };
+    // key of the host at table position `pos` for a request of g GPUs: A + g * B (low bits = host id)
+    auto key_at = [&](unsigned int pos, int g) -> unsigned int {
+        const uint2 ab = __ldg(reinterpret_cast<const uint2 *>(p.ab) + row + pos);
+        return ab.x + (unsigned int)g * ab.y;
+    };
 
     // Two-word form of each request. With two levels it is needed only in the chunks that pass
     // the first level, and is kept in local memory (indexed dynamically below) so that the pair
     // loop has its registers for first-level words; otherwise it stays in registers.
     unsigned long long rq_keep[Q];
     unsigned int r1[TWO_LEVELS ? Q : 1];   // first-level word
-    unsigned int best[3 * Q];  // positions of the best three: [0, Q) best, [Q, 2Q) second, [2Q, 3Q) third
+    constexpr bool by_group = BY_GROUP;
+    unsigned int best[3 * Q];  // the best three, [0, Q) best, [Q, 2Q) second, [2Q, 3Q) third: positions, or
+                               // (by_group) keys over all groups
+    unsigned int fits[BY_GROUP ? 3 * Q : 1];  // by_group: positions of the first three hosts of the current group that fit
     unsigned int field[Q];     // rank field of each request after an update
     unsigned int opened[Q];    // position of the third host the opening found (kNone: fewer than three)
 
-    // ---- opening: the first hosts of the slice, exactly, eight at a time ----
-    const int open_pos = tile_begin * T;
-    unsigned int o1[Q], o2[Q], o3[Q];
-    int4 ask[Q];
 #pragma unroll
     for (int q = 0; q < Q; ++q) {
-        ask[q] = load_request(q);
-        o1[q] = kNone; o2[q] = kNone; o3[q] = kNone;
+        best[q] = kNone; best[Q + q] = kNone; best[2 * Q + q] = kNone;
     }
+    bool words_built = false;
+
+    // slice after slice: the opening, then the pair loop over the slice's tiles. (A block with one
+    // slice has the same host range in every pass, computed once by the caller; its loop below runs
+    // once.)
+    int sl = slice_first;
+    do {
+        const SliceRange sr = BY_GROUP ? slice_range(p, n, sl) : own_slice;
+        if (BY_GROUP && sr.hi <= sr.lo) continue;
+        // ---- opening: the first hosts of the slice, exactly, eight at a time ----
+        const int open_pos = sr.real_lo;
+        const int open_end = min(sr.real_lo + kOpeningHosts, sr.real_hi);
+        {
+            unsigned int o1[Q], o2[Q], o3[Q];
+            int4 ask[Q];
+#pragma unroll
+            for (int q = 0; q < Q; ++q) {
+                ask[q] = load_request(q);
+                o1[q] = kNone; o2[q] = kNone; o3[q] = kNone;
+            }
 #pragma unroll 1
-    for (int base = 0; base < kOpeningHosts; base += 8) {
-        bool need = false;
+            for (int base = 0; base < kOpeningHosts; base += 8) {
+                bool need = false;
 #pragma unroll
-        for (int q = 0; q < Q; ++q) need |= o3[q] == kNone;
-        if (!need) break;
-        int4 f[8];
+                for (int q = 0; q < Q; ++q) need |= o3[q] == kNone;
+                if (!need) break;
+                int4 f[8];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) f[u] = __ldg(p.feas + row + open_pos + base + u);
+                for (int u = 0; u < 8; ++u)   // hosts past the end of a group take nothing (ordinary slices have 32 hosts or more)
+                    f[u] = (!BY_GROUP || open_pos + base + u < open_end) ? __ldg(p.feas + row + open_pos + base + u)
+                                                                          : make_int4(-1, 0, 0, 0);
 #pragma unroll
-        for (int q = 0; q < Q; ++q)
+                for (int q = 0; q < Q; ++q)
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const bool ok = (ask[q].x <= f[u].x) & (ask[q].y <= f[u].y) & (ask[q].z <= f[u].z) & (ask[q].w <= f[u].w);
-                // positions come in ascending order: a fitting host takes the first free slot
-                const unsigned int pos = (unsigned int)(open_pos + base + u);
-                const bool take3 = ok & (o2[q] != kNone) & (o3[q] == kNone);
-                const bool take2 = ok & (o1[q] != kNone) & (o2[q] == kNone);
-                const bool take1 = ok & (o1[q] == kNone);
-                o3[q] = take3 ? pos : o3[q];
-                o2[q] = take2 ? pos : o2[q];
-                o1[q] = take1 ? pos : o1[q];
+                    for (int u = 0; u < 8; ++u) {
+                        const bool ok = (ask[q].x <= f[u].x) & (ask[q].y <= f[u].y) & (ask[q].z <= f[u].z) & (ask[q].w <= f[u].w);
+                        // positions come in ascending order: a fitting host takes the first free slot
+                        const unsigned int pos = (unsigned int)(open_pos + base + u);
+                        const bool take3 = ok & (o2[q] != kNone) & (o3[q] == kNone);
+                        const bool take2 = ok & (o1[q] != kNone) & (o2[q] == kNone);
+                        const bool take1 = ok & (o1[q] == kNone);
+                        o3[q] = take3 ? pos : o3[q];
+                        o2[q] = take2 ? pos : o2[q];
+                        o1[q] = take1 ? pos : o1[q];
+                    }
             }
-    }
-#pragma unroll
-    for (int q = 0; q < Q; ++q) {
-        const int4 r = ask[q];
-        // an ask above every host's capacity in some resource fits nowhere either: encode both
-        // cases as a GPU ask above every gmax and keep the other fields inside their widths
-        const bool bad = (r.x > p.rank.fmax[0]) | (r.y > p.rank.fmax[1]) | (r.z > p.rank.fmax[2]) |
-                         (r.w > p.rank.fmax[3]);
-        const unsigned int val[4] = {bad ? (unsigned int)p.rank.fmax[0] + 2u : (unsigned int)r.x + 1u,
-                                     bad ? 0u : (unsigned int)r.y, bad ? 0u : (unsigned int)r.z,
-                                     bad ? 0u : (unsigned int)r.w};
-        unsigned int w0 = 0u, w1 = 0u, l1 = 0u;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const unsigned int piece = (val[k] >> p.rank.fdrop[k]) << p.rank.fshift[k];
-            if (p.rank.fword[k]) w1 |= piece; else w0 |= piece;
-            l1 |= (val[k] >> p.rank.l1_drop[k]) << p.rank.l1_shift[k];
-        }
-        // rank field from the opening's third host (0 = every rank passes)
-        const unsigned int fld = o3[q] == kNone ? 0u : p.rank.rank_top + 1u - o3[q];
-        rq_keep[q] = ((unsigned long long)w0 | ((unsigned long long)w1 << 32)) | ((unsigned long long)fld << rank_shift);
-        if constexpr (TWO_LEVELS) r1[q] = l1 | (fld << p.rank.l1_shift[4]);
-        const bool keeper = sub == 0;   // one lane of the group carries the opening's finds to the merge
-        best[q] = keeper ? o1[q] : kNone; best[Q + q] = keeper ? o2[q] : kNone; best[2 * Q + q] = keeper ? o3[q] : kNone;
-        field[q] = fld;
-        opened[q] = o3[q];
-    }
-
-    for (int t = tile_begin; t < tile_end; ++t, ++ring_pos) {
-        const uint32_t s = ring_pos % kStages;
-        const uint32_t parity = (ring_pos / kStages) & 1u;
-        if (!mbar_wait(full_bar + 8u * s, parity, abort_flag)) return false;
-        const unsigned long long *R = reinterpret_cast<const unsigned long long *>(stages + (size_t)s * stage_bytes);
-        const unsigned int *R1 = reinterpret_cast<const unsigned int *>(R + T);
-        const int pos0 = t * T;
-        int hosts = p.Hpad - pos0;
-        if (hosts > T) hosts = T;
-        const int n_groups = hosts >> 2;   // groups of four hosts in this tile (hosts is a multiple of 32)
-
-        // two-word test of host group gi (hosts 4 gi .. 4 gi + 3 of the tile) against the Q
-        // requests, then the exact part
-        auto group2 = [&](int gi) {
-            unsigned long long h[4];
-            {
-                const ulonglong2 a = *reinterpret_cast<const ulonglong2 *>(R + 4 * gi);
-                const ulonglong2 b = *reinterpret_cast<const ulonglong2 *>(R + 4 * gi + 2);
-                h[0] = a.x; h[1] = a.y; h[2] = b.x; h[3] = b.y;
-            }
-            unsigned long long rq[Q];
-#pragma unroll
-            for (int q = 0; q < Q; ++q) rq[q] = rq_keep[q];
-            if (!ranked_chunk_any_pass<Q, 4>(rq, h, guards)) return;
-            // rare. Which pairs passed (bit 4 q + u), with static register indices ...
-            unsigned int passed = 0u;
-#pragma unroll
-            for (int q = 0; q < Q; ++q)
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const unsigned long long d = h[u] - rq[q];
-                    const unsigned int fell = ~((unsigned int)d & (unsigned int)(d >> 32)) & guards;
-                    passed |= (fell == 0u ? 1u : 0u) << (q * 4 + u);
-                }
-            // ... then one pair after the other: exact test against the request as given; the
-            // best-three arrays are indexed dynamically here and therefore live in local memory,
-            // which keeps their 3 * Q registers out of the pair loop
-            unsigned int touched = 0u;
-            while (passed) {
-                const int bit = __ffs(passed) - 1;
-                passed &= passed - 1u;
-                const int q = bit >> 2, u = bit & 3;
-                const unsigned int pos = (unsigned int)(pos0 + 4 * gi + u);
-                const int4 r = load_request(q);
-                const int4 f = __ldg(p.feas + row + pos);
-                if ((r.x <= f.x) & (r.y <= f.y) & (r.z <= f.z) & (r.w <= f.w)) {
-                    unsigned int a1 = best[q], a2 = best[Q + q], a3 = best[2 * Q + q];
-                    insert3(a1, a2, a3, pos);
-                    best[q] = a1; best[Q + q] = a2; best[2 * Q + q] = a3;
-                    const unsigned int third = min(a3, opened[q]);   // the other lanes' opening finds count too
-                    field[q] = third == kNone ? 0u : p.rank.rank_top + 1u - third;
-                    if constexpr (TWO_LEVELS)
-                        rq_keep[q] = (rq_keep[q] & ~rank_mask) | ((unsigned long long)field[q] << rank_shift);
-                    touched = 1u;
-                }
-            }
-            if (touched) {
+            if (!BY_GROUP || !words_built) {
+                // the packed forms of the requests, once per pass (rank fields 0 so far)
+                words_built = true;
 #pragma unroll
                 for (int q = 0; q < Q; ++q) {
-                    if constexpr (TWO_LEVELS) r1[q] = (r1[q] & ~p.rank.l1_rank_mask) | (field[q] << p.rank.l1_shift[4]);
-                    else rq_keep[q] = (rq_keep[q] & ~rank_mask) | ((unsigned long long)field[q] << rank_shift);
+                    const int4 r = ask[q];
+                    // an ask above every host's capacity in some resource fits nowhere either: encode both
+                    // cases as a GPU ask above every gmax and keep the other fields inside their widths
+                    const bool bad = (r.x > p.rank.fmax[0]) | (r.y > p.rank.fmax[1]) | (r.z > p.rank.fmax[2]) |
+                                     (r.w > p.rank.fmax[3]);
+                    const unsigned int val[4] = {bad ? (unsigned int)p.rank.fmax[0] + 2u : (unsigned int)r.x + 1u,
+                                                 bad ? 0u : (unsigned int)r.y, bad ? 0u : (unsigned int)r.z,
+                                                 bad ? 0u : (unsigned int)r.w};
+                    unsigned int w0 = 0u, w1 = 0u, l1 = 0u;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const unsigned int piece = (val[k] >> p.rank.fdrop[k]) << p.rank.fshift[k];
+                        if (p.rank.fword[k]) w1 |= piece; else w0 |= piece;
+                        l1 |= (val[k] >> p.rank.l1_drop[k]) << p.rank.l1_shift[k];
+                    }
+                    rq_keep[q] = (unsigned long long)w0 | ((unsigned long long)w1 << 32);
+                    if constexpr (TWO_LEVELS) r1[q] = l1;
                 }
             }
-        };
-
-        // this lane's host groups: sub, sub + L, ...; the opening has dealt with the slice's first ones
-        int g = sub;
-        if (t == tile_begin)
-            while (g < kOpeningHosts / 4) g += L;
-        if constexpr (TWO_LEVELS) {
-            // first level of W / 4 host groups (g0, g0 + L, ...) against the Q requests
-            auto chunk1 = [&](auto width, int g0) {
-                constexpr int W = decltype(width)::value;
-                unsigned int h1[W];
+            const bool keeper = sub == 0;   // one lane of the group carries the opening's finds to the merge
 #pragma unroll
-                for (int v = 0; v < W / 4; ++v) {
-                    const uint4 a = *reinterpret_cast<const uint4 *>(R1 + 4 * (g0 + v * L));
-                    h1[4 * v] = a.x; h1[4 * v + 1] = a.y; h1[4 * v + 2] = a.z; h1[4 * v + 3] = a.w;
+            for (int q = 0; q < Q; ++q) {
+                // rank field from the opening's third host (0 = every rank passes)
+                const unsigned int fld = o3[q] == kNone ? 0u : p.rank.rank_top + 1u - o3[q];
+                rq_keep[q] = (rq_keep[q] & ~rank_mask) | ((unsigned long long)fld << rank_shift);
+                if constexpr (TWO_LEVELS) r1[q] = (r1[q] & ~p.rank.l1_rank_mask) | (fld << p.rank.l1_shift[4]);
+                field[q] = fld;
+                opened[q] = o3[q];
+                if constexpr (!BY_GROUP) {
+                    best[q] = keeper ? o1[q] : kNone; best[Q + q] = keeper ? o2[q] : kNone; best[2 * Q + q] = keeper ? o3[q] : kNone;
+                } else {
+                    fits[q] = keeper ? o1[q] : kNone; fits[Q + q] = keeper ? o2[q] : kNone; fits[2 * Q + q] = keeper ? o3[q] : kNone;
+                    if (keeper && o1[q] != kNone) {
+                        unsigned int a1 = best[q], a2 = best[Q + q], a3 = best[2 * Q + q];
+                        insert3(a1, a2, a3, key_at(o1[q], ask[q].x));
+                        if (o2[q] != kNone) insert3(a1, a2, a3, key_at(o2[q], ask[q].x));
+                        if (o3[q] != kNone) insert3(a1, a2, a3, key_at(o3[q], ask[q].x));
+                        best[q] = a1; best[Q + q] = a2; best[2 * Q + q] = a3;
+                    }
                 }
-                unsigned int groups_passed = ranked_l1_chunk_groups_passed<Q, W>(r1, h1, guards1);
-                // second level only for the groups of four hosts in which a pair passed
-                while (groups_passed) {
-                    const int v = __ffs(groups_passed) - 1;
-                    groups_passed &= groups_passed - 1u;
-                    group2(g0 + v * L);
+            }
+        }
+
+        for (int pos0 = sr.lo; pos0 < sr.hi; pos0 += T, ++ring_pos) {
+            const uint32_t s = ring_pos % kStages;
+            const uint32_t parity = (ring_pos / kStages) & 1u;
+            if (!mbar_wait(full_bar + 8u * s, parity, abort_flag)) return false;
+            const unsigned long long *R = reinterpret_cast<const unsigned long long *>(stages + (size_t)s * stage_bytes);
+            const unsigned int *R1 = reinterpret_cast<const unsigned int *>(R + T);
+            int hosts = sr.hi - pos0;
+            if (hosts > T) hosts = T;
+            const int n_groups = hosts >> 2;   // groups of four hosts in this tile (hosts is a multiple of 4)
+
+            // two-word test of host group gi (hosts 4 gi .. 4 gi + 3 of the tile) against the Q
+            // requests, then the exact part
+            auto group2 = [&](int gi) {
+                unsigned long long h[4];
+                {
+                    const ulonglong2 a = *reinterpret_cast<const ulonglong2 *>(R + 4 * gi);
+                    const ulonglong2 b = *reinterpret_cast<const ulonglong2 *>(R + 4 * gi + 2);
+                    h[0] = a.x; h[1] = a.y; h[2] = b.x; h[3] = b.y;
+                }
+                unsigned long long rq[Q];
+#pragma unroll
+                for (int q = 0; q < Q; ++q) rq[q] = rq_keep[q];
+                if (!ranked_chunk_any_pass<Q, 4>(rq, h, guards)) return;
+                // rare. Which pairs passed (bit 4 q + u), with static register indices ...
+                unsigned int passed = 0u;
+#pragma unroll
+                for (int q = 0; q < Q; ++q)
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const unsigned long long d = h[u] - rq[q];
+                        const unsigned int fell = ~((unsigned int)d & (unsigned int)(d >> 32)) & guards;
+                        passed |= (fell == 0u ? 1u : 0u) << (q * 4 + u);
+                    }
+                // ... then one pair after the other: exact test against the request as given; the
+                // best-three arrays are indexed dynamically here and therefore live in local memory,
+                // which keeps their registers out of the pair loop
+                unsigned int touched = 0u;
+                while (passed) {
+                    const int bit = __ffs(passed) - 1;
+                    passed &= passed - 1u;
+                    const int q = bit >> 2, u = bit & 3;
+                    const unsigned int pos = (unsigned int)(pos0 + 4 * gi + u);
+                    // the opening has dealt with the group's first hosts; what was staged beyond the
+                    // group's ends belongs to a neighbouring group. (Ordinary slices are whole tiles
+                    // and the pair loop starts right behind the opening: nothing to leave out.)
+                    if constexpr (BY_GROUP)
+                        if ((int)pos < open_end || (int)pos >= sr.real_hi) continue;
+                    const int4 r = load_request(q);
+                    const int4 f = __ldg(p.feas + row + pos);
+                    if ((r.x <= f.x) & (r.y <= f.y) & (r.z <= f.z) & (r.w <= f.w)) {
+                        unsigned int a1 = best[q], a2 = best[Q + q], a3 = best[2 * Q + q];
+                        insert3(a1, a2, a3, by_group ? key_at(pos, r.x) : pos);
+                        best[q] = a1; best[Q + q] = a2; best[2 * Q + q] = a3;
+                        unsigned int f3 = a3;
+                        if constexpr (BY_GROUP) {
+                            unsigned int f1 = fits[q], f2 = fits[Q + q];
+                            f3 = fits[2 * Q + q];
+                            insert3(f1, f2, f3, pos);
+                            fits[q] = f1; fits[Q + q] = f2; fits[2 * Q + q] = f3;
+                        }
+                        const unsigned int third = min(f3, opened[q]);   // the other lanes' opening finds count too
+                        field[q] = third == kNone ? 0u : p.rank.rank_top + 1u - third;
+                        if constexpr (TWO_LEVELS)
+                            rq_keep[q] = (rq_keep[q] & ~rank_mask) | ((unsigned long long)field[q] << rank_shift);
+                        touched = 1u;
+                    }
+                }
+                if (touched) {
+#pragma unroll
+                    for (int q = 0; q < Q; ++q) {
+                        if constexpr (TWO_LEVELS) r1[q] = (r1[q] & ~p.rank.l1_rank_mask) | (field[q] << p.rank.l1_shift[4]);
+                        else rq_keep[q] = (rq_keep[q] & ~rank_mask) | ((unsigned long long)field[q] << rank_shift);
+                    }
                 }
             };
-            for (; g + 3 * L < n_groups; g += 4 * L) chunk1(std::integral_constant<int, 16>{}, g);
-            for (; g < n_groups; g += L) chunk1(std::integral_constant<int, 4>{}, g);
-        } else {
-            for (; g < n_groups; g += L) group2(g);
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty_bar + 8u * s);
-    }
 
-    // merge the L lanes of a group (positions are unique)
+            // this lane's host groups: sub, sub + L, ...; the groups that lie entirely inside the
+            // opening's range are left out
+            int g = sub;
+            if (pos0 == sr.lo)
+                while (g < ((open_end - sr.lo) >> 2)) g += L;
+            if constexpr (TWO_LEVELS) {
+                // first level of W / 4 host groups (g0, g0 + L, ...) against the Q requests
+                auto chunk1 = [&](auto width, int g0) {
+                    constexpr int W = decltype(width)::value;
+                    unsigned int h1[W];
+#pragma unroll
+                    for (int v = 0; v < W / 4; ++v) {
+                        const uint4 a = *reinterpret_cast<const uint4 *>(R1 + 4 * (g0 + v * L));
+                        h1[4 * v] = a.x; h1[4 * v + 1] = a.y; h1[4 * v + 2] = a.z; h1[4 * v + 3] = a.w;
+                    }
+                    unsigned int groups_passed = ranked_l1_chunk_groups_passed<Q, W>(r1, h1, guards1);
+                    // second level only for the groups of four hosts in which a pair passed
+                    while (groups_passed) {
+                        const int v = __ffs(groups_passed) - 1;
+                        groups_passed &= groups_passed - 1u;
+                        group2(g0 + v * L);
+                    }
+                };
+                for (; g + 3 * L < n_groups; g += 4 * L) chunk1(std::integral_constant<int, 16>{}, g);
+                for (; g < n_groups; g += L) chunk1(std::integral_constant<int, 4>{}, g);
+            } else {
+                for (; g < n_groups; g += L) group2(g);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty_bar + 8u * s);
+        }
+    } while (BY_GROUP && ++sl < slice_last);
+
+    // merge the L lanes of a group (keys and positions are unique, so the order of merging does not matter)
     unsigned int t1[Q], t2[Q], t3[Q];
 #pragma unroll
     for (int q = 0; q < Q; ++q) { t1[q] = best[q]; t2[q] = best[Q + q]; t3[q] = best[2 * Q + q]; }
@@ -729,13 +832,13 @@ __device__ __forceinline__ bool run_pass_ranked(const PlaceParams &p, unsigned c
             const int idx = q * kGroups + grp;
             if (idx >= count) continue;
             const long long r = first + idx;
-            // position -> key (its low bits are the host id; all hosts share the key slope, so
-            // the intercepts order like the keys)
-            const unsigned int k1 = t1[q] == kNone ? kNone : __ldg(&AB[t1[q]].x);
-            const unsigned int k2 = t2[q] == kNone ? kNone : __ldg(&AB[t2[q]].x);
-            const unsigned int k3 = t3[q] == kNone ? kNone : __ldg(&AB[t3[q]].x);
+            // single slice: position -> key (its low bits are the host id; all hosts of the slice
+            // share the key slope, so the intercepts order like the keys)
+            const unsigned int k1 = by_group || t1[q] == kNone ? t1[q] : __ldg(&AB[t1[q]].x);
+            const unsigned int k2 = by_group || t2[q] == kNone ? t2[q] : __ldg(&AB[t2[q]].x);
+            const unsigned int k3 = by_group || t3[q] == kNone ? t3[q] : __ldg(&AB[t3[q]].x);
             if (p.K > 1) {
-                unsigned int *cand = reinterpret_cast<unsigned int *>(p.cand) + ((long long)slice * p.n_req + (r - p.first_req)) * 3;
+                unsigned int *cand = reinterpret_cast<unsigned int *>(p.cand) + ((long long)slice_first * p.n_req + (r - p.first_req)) * 3;
                 cand[0] = k1; cand[1] = k2; cand[2] = k3;
             } else {
                 int32_t *o = p.out_hosts + r * 3;
@@ -777,8 +880,10 @@ place_kernel(const __grid_constant__ PlaceParams p)
 
     const int slice = blockIdx.x / p.req_ctas;
     const int cr = blockIdx.x % p.req_ctas;
-    const int tile_begin = (int)((long long)p.tiles_total * slice / p.K);
-    const int tile_end = (int)((long long)p.tiles_total * (slice + 1) / p.K);
+    // a block has one host slice, except for grouped tables in the ranked form, whose blocks walk
+    // all GPU-count groups (K = 1 there)
+    const int slice_first = mode_ranked_by_group(MODE) ? 0 : slice;
+    const int slice_last = mode_ranked_by_group(MODE) ? kGroupSlices : slice + 1;
     PassList passes;
     block_request_range(p, cr, passes.cursor, passes.hi);
     passes.B = p.B;
@@ -794,9 +899,13 @@ place_kernel(const __grid_constant__ PlaceParams p)
         const uint32_t stage0 = smem_addr(smem);
         uint32_t issued = 0;
         bool ok = true;
+        SliceRange copy_slice = {0, 0, 0, 0};
+        if (!mode_ranked_by_group(MODE)) copy_slice = slice_range(p, 0, slice);
         while (ok && passes.next(n, first, count, q)) {
             const size_t row = (size_t)n * p.Hpad;
-            for (int t = tile_begin; t < tile_end; ++t, ++issued) {
+            for (int sl = slice_first; ok && sl < slice_last; ++sl) {
+            const SliceRange sr = mode_ranked_by_group(MODE) ? slice_range(p, n, sl) : copy_slice;
+            for (int pos0 = sr.lo; pos0 < sr.hi; pos0 += T, ++issued) {
                 const uint32_t s = issued % kStages;
                 if (issued >= (uint32_t)kStages) {
                     const uint32_t parity = ((issued / kStages) - 1u) & 1u;
@@ -805,30 +914,32 @@ place_kernel(const __grid_constant__ PlaceParams p)
                         break;
                     }
                 }
-                int hosts = p.Hpad - t * T;
+                int hosts = sr.hi - pos0;
                 if (hosts > T) hosts = T;
                 const uint32_t dst = stage0 + s * stage_bytes;
                 if (mode_is_ranked(MODE)) {
+                    // pos0 and hosts are multiples of four: 16-byte aligned sources and sizes
                     const uint32_t bytes = (uint32_t)hosts * 8u;
-                    const uint32_t bytes1 = MODE == MODE_RANKED2 ? (uint32_t)hosts * 4u : 0u;
+                    const uint32_t bytes1 = mode_ranked_two_levels(MODE) ? (uint32_t)hosts * 4u : 0u;
                     mbar_arrive_expect_tx(full_bar + 8u * s, bytes + bytes1);
-                    bulk_copy_g2s(dst, p.rk + row + (size_t)t * T, bytes, full_bar + 8u * s);
-                    if (MODE == MODE_RANKED2)
-                        bulk_copy_g2s(dst + (uint32_t)T * 8u, p.rk1 + row + (size_t)t * T, bytes1, full_bar + 8u * s);
+                    bulk_copy_g2s(dst, p.rk + row + pos0, bytes, full_bar + 8u * s);
+                    if (mode_ranked_two_levels(MODE))
+                        bulk_copy_g2s(dst + (uint32_t)T * 8u, p.rk1 + row + pos0, bytes1, full_bar + 8u * s);
                 } else if (kPacked) {
                     const uint32_t bytes = (uint32_t)hosts * 16u;
                     mbar_arrive_expect_tx(full_bar + 8u * s, bytes);
-                    bulk_copy_g2s(dst, p.pk + row + (size_t)t * T, bytes, full_bar + 8u * s);
+                    bulk_copy_g2s(dst, p.pk + row + pos0, bytes, full_bar + 8u * s);
                 } else {
                     const uint32_t pair_bytes = (uint32_t)kRecord - 16u;
                     const uint32_t bytes_f = (uint32_t)hosts * 16u;
                     const uint32_t bytes_k = (uint32_t)hosts * pair_bytes;
                     mbar_arrive_expect_tx(full_bar + 8u * s, bytes_f + bytes_k);
-                    bulk_copy_g2s(dst, p.feas + row + (size_t)t * T, bytes_f, full_bar + 8u * s);
+                    bulk_copy_g2s(dst, p.feas + row + pos0, bytes_f, full_bar + 8u * s);
                     bulk_copy_g2s(dst + (uint32_t)T * 16u,
-                                  static_cast<const unsigned char *>(p.ab) + (row + (size_t)t * T) * pair_bytes,
+                                  static_cast<const unsigned char *>(p.ab) + (row + (size_t)pos0) * pair_bytes,
                                   bytes_k, full_bar + 8u * s);
                 }
+            }
             }
         }
         if (!ok) {
@@ -849,11 +960,16 @@ place_kernel(const __grid_constant__ PlaceParams p)
     // ---- compute threads ----
     uint32_t ring_pos = 0;
     bool ok = true;
+    // an ordinary slice (whole tiles) is the same for every snapshot
+    SliceRange own_slice = {0, 0, 0, 0};
+    if (!mode_ranked_by_group(MODE)) own_slice = slice_range(p, 0, slice);
+    const int tile_begin = own_slice.lo / T, tile_end = (own_slice.hi + T - 1) / T;
+    (void)tile_begin; (void)tile_end;
     while (ok && passes.next(n, first, count, q)) {
 #define NBOS_PASS(QV)                                                                                 \
     if constexpr (mode_is_ranked(MODE))                                                               \
-        ok = run_pass_ranked<QV, L, MODE == MODE_RANKED2>(p, smem, stage_bytes, full_bar, empty_bar, abort_flag, ring_pos,  \
-                                    tile_begin, tile_end, slice, first, count, n);                    \
+        ok = run_pass_ranked<QV, L, mode_ranked_two_levels(MODE), mode_ranked_by_group(MODE)>(p, smem, stage_bytes, full_bar, empty_bar, abort_flag, ring_pos,  \
+                                    slice_first, slice_last, own_slice, first, count, n);             \
     else                                                                                              \
         ok = run_pass<QV, L, MODE>(p, smem, stage_bytes, full_bar, empty_bar, abort_flag, ring_pos,   \
                                    tile_begin, tile_end, slice, first, count)
@@ -1044,6 +1160,8 @@ KernelFn pick_kernel(int mode, int L)
         case MODE_GROUPED2: return pick_kernel_l<MODE_GROUPED2>(L);
         case MODE_RANKED: return pick_kernel_l<MODE_RANKED>(L);
         case MODE_RANKED2: return pick_kernel_l<MODE_RANKED2>(L);
+        case MODE_RANKED_GROUPS: return pick_kernel_l<MODE_RANKED_GROUPS>(L);
+        case MODE_RANKED2_GROUPS: return pick_kernel_l<MODE_RANKED2_GROUPS>(L);
     }
     return nullptr;
 }
@@ -1079,7 +1197,11 @@ int kernel_occupancy(KernelFn fn, int device, size_t smem, int *per_sm)
 int snapshot_mode(const nbos_snapshot *s, int forced)
 {
     if (s->key.key_bits == 64) return MODE_KEY64;
-    if ((forced == 0 || forced == 5) && s->rank.enabled) return (forced == 0 && s->rank.l1_enabled) ? MODE_RANKED2 : MODE_RANKED;
+    if ((forced == 0 || forced == 5) && s->rank.enabled) {
+        const bool two = forced == 0 && s->rank.l1_enabled;
+        if (s->key.grouped) return two ? MODE_RANKED2_GROUPS : MODE_RANKED_GROUPS;
+        return two ? MODE_RANKED2 : MODE_RANKED;
+    }
     if (forced == 1 || !s->pack.enabled) return MODE_PLAIN;
     const bool two = s->pack.guards != s->pack.guards1;
     if ((forced == 0 || forced == 4) && s->key.grouped) return two ? MODE_GROUPED2 : MODE_GROUPED;
@@ -1108,6 +1230,7 @@ void fill_params(PlaceParams &p, const nbos_snapshot *s, const int32_t *d_reques
     p.first_req = 0;
     p.n_req = p.total;
     p.per_snapshot = 0;
+    p.group_bounds = nullptr;
     p.N = s->N;
     p.Hpad = s->Hpad;
     p.id_mask = (1u << s->key.bits_id) - 1u;
@@ -1128,6 +1251,7 @@ int make_plan(const nbos_snapshot *s, long long total, long long batch, const nb
               bool whole_batch, LaunchPlan &plan)
 {
     const int mode = snapshot_mode(s, c.pair_mode);
+    const int host_div = 1;
     const int record = mode_record_bytes(mode);
     const int max_q_kernel = mode_max_q(mode);
 
@@ -1157,7 +1281,7 @@ int make_plan(const nbos_snapshot *s, long long total, long long batch, const nb
     int blocks_per_sm = per_sm;
     plan.per_snapshot = 0;
     {
-        const bool two_level = mode == MODE_RANKED2;
+        const bool two_level = mode_ranked_two_levels(mode);
         const double pair_cost = two_level ? 1.8 : (mode_is_sorted(mode) || mode_is_ranked(mode)) ? 3.0 : mode_is_grouped(mode) ? 3.3
                                  : mode_is_static(mode) ? 4.0 : mode_is_packed(mode) ? 5.0 : mode == MODE_PLAIN ? 7.0 : 12.0;
         // The two-level ranked form has a cheap pair step and a dearer start of every request (its
@@ -1174,12 +1298,13 @@ int make_plan(const nbos_snapshot *s, long long total, long long batch, const nb
         for (int cand = 1, lg = 0; cand <= 32; cand <<= 1, ++lg) {
             if (c.lanes_per_request && cand != c.lanes_per_request) continue;
             const long long groups = kComputeThreads / cand;
-            const double per_host = (double)s->Hpad / cand;
+            const double per_host = (double)s->Hpad / host_div / cand;
             for (int j = per_sm; j >= 1; --j) {
                 const long long slots = (long long)s->sm_count * j;
-                long long ctas = (total + groups - 1) / groups;
+                // (grouped ranked form: every request is looked at by host_div blocks)
+                long long ctas = (total * host_div + groups - 1) / groups;
                 if (ctas > slots) ctas = slots;
-                long long n_req = (total + ctas - 1) / ctas;
+                long long n_req = (total * host_div + ctas - 1) / ctas;
                 n_req = (n_req + 31) / 32 * 32;
                 auto pass = [&](int qq) {
                     return kPassCost + qq * kRequestCost + per_host * (kHostCost + pair_cost * qq) + lg * qq * kMergeCost;
@@ -1258,6 +1383,9 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
     nbos_launch_config c = {};
     if (cfg) c = *cfg;
     if (c.reserved != 0) return fail(NBOS_ERR_INVALID_ARG, "launch config: reserved field must be 0");
+    // The ranked form of a grouped table slices the hosts by GPU-count group; a caller who asks for
+    // a host split of his own gets the form that can take any split.
+    if (s->key.grouped && c.host_split > 0 && c.pair_mode == 0) c.pair_mode = 4;
     if (c.first_fit < 0 || c.first_fit > 1) return fail(NBOS_ERR_INVALID_ARG, "first_fit must be 0 or 1");
     if (c.lanes_per_request && !(is_pow2(c.lanes_per_request) && c.lanes_per_request <= 32))
         return fail(NBOS_ERR_INVALID_ARG, "lanes_per_request must be 1,2,4,8,16 or 32");
@@ -1302,17 +1430,22 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
     // Hosts are cut into slices only when the batch is so small that even a warp per request
     // leaves SMs without a block.
     const long long one_block_per_sm = (long long)s->sm_count * kComputeThreads;
+    const bool by_group = mode_ranked_by_group(mode);
     int K = c.host_split;
-    if (!K) {
-        K = 1;
-        if (total * 32 < one_block_per_sm && !c.lanes_per_request) {
-            const long long k = (one_block_per_sm + total * 32 - 1) / (total * 32);
-            K = (int)(k < tiles_total ? k : tiles_total);
+    if (by_group) {
+        K = 1;   // a block walks all GPU-count groups itself
+    } else {
+        if (!K) {
+            K = 1;
+            if (total * 32 < one_block_per_sm && !c.lanes_per_request) {
+                const long long k = (one_block_per_sm + total * 32 - 1) / (total * 32);
+                K = (int)(k < tiles_total ? k : tiles_total);
+            }
         }
+        if (K > tiles_total) K = tiles_total;
+        if (K < 1) K = 1;
     }
-    if (K > tiles_total) K = tiles_total;
-    if (K < 1) K = 1;
-    const int L = (K > 1 && !c.lanes_per_request) ? 32 : plan.L;
+    const int L = (K > 1 && !by_group && !c.lanes_per_request) ? 32 : plan.L;
 
     int max_q = c.requests_per_lane ? c.requests_per_lane : max_q_kernel;
     if (max_q > max_q_kernel) max_q = max_q_kernel;
@@ -1325,7 +1458,7 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
 
     const int groups = kComputeThreads / L;
     long long req_ctas = (total + groups - 1) / groups;  // at least one request per group
-    if (per_sm > plan.blocks_per_sm && K == 1) per_sm = plan.blocks_per_sm;
+    if (per_sm > plan.blocks_per_sm && (K == 1 || by_group)) per_sm = plan.blocks_per_sm;
     long long cap = (long long)s->sm_count * per_sm / K;
     if (cap < 1) cap = 1;
     if (c.grid_blocks) cap = c.grid_blocks;
@@ -1336,6 +1469,7 @@ int launch_place(const nbos_snapshot *s, const int32_t *d_requests, int64_t batc
     PlaceParams p;
     fill_params(p, s, d_requests, batch, d_out_hosts, d_out_found);
     p.per_snapshot = per_snapshot;
+    p.group_bounds = by_group ? s->d_group_bounds : nullptr;
     p.first_req = range_first;
     p.n_req = range_count;
     p.tile_hosts = T;
@@ -1416,7 +1550,9 @@ int launch_place_static(const nbos_snapshot *s, const int32_t *d_requests, int64
     NBOS_CUDA_TRY(cudaGetDevice(&device));
     if (device != s->device)
         return fail(NBOS_ERR_INVALID_ARG, "snapshot was created on device %d, current device is %d", s->device, device);
-    const int mode = snapshot_mode(s, 0);
+    // (a grouped table's ranked form slices the hosts its own way; this entry point's slices are
+    // the caller's, so it takes the grouped form that works with any slice)
+    const int mode = snapshot_mode(s, s->key.grouped ? 4 : 0);
     const bool k64 = mode == MODE_KEY64;
     const int key_bytes = k64 ? 8 : 4;
     const int record = mode_record_bytes(mode);

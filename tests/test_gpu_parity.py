@@ -257,9 +257,11 @@ def test_ranked_form_coarse_fields(nb):
     for flags in (0, 1):
         got, ref = both(nb, w3, flags=flags)
         assert_same(got, ref, f"crowded VRAM flags={flags}")
-    # (d) mixed GPU counts have no ranked form (hosts rank differently for different asks)
+    # (d) mixed GPU counts: hosts rank differently for different asks, but the same inside one GPU
+    # count; the ranked form then works group by group (the groups are the host slices)
     s = nb.snapshot_from_workload(W.mixed_gpu_cluster(300, 100, seed=8))
-    assert s.info().ranked == 0
+    info = s.info()
+    assert (info.ranked, info.grouped, info.static_key) == (1, 1, 0)
     nb.nbos_snapshot_destroy(s)
 
 
