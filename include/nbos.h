@@ -343,13 +343,14 @@ int nbos_select_executors(const nbos_cluster_state *state, const int32_t *reques
  * and the other capacities stay as they are. Snapshots are independent and run in parallel; the
  * snapshot object itself is not modified.
  *   snap            must have been created with NBOS_ROOM_FOR_COMMITS; at most
- *                   NBOS_SEQUENTIAL_MAX_HOSTS hosts (the evolving state lives on one SM);
+ *                   NBOS_SEQUENTIAL_MAX_HOSTS hosts (the evolving state lives on one SM up to
+ *                   8,192 hosts, on the 2 to 8 SMs of a thread-block cluster beyond that);
  *                   otherwise INVALID_ARG / RANGE
  *   requests, out_hosts, out_found   as for nbos_place_batch
  *   out_subscribed  DEVICE [N * H] int32 or NULL: S of every host after the last request
  * Asynchronous on `cuda_stream`.
  */
-#define NBOS_SEQUENTIAL_MAX_HOSTS 8192
+#define NBOS_SEQUENTIAL_MAX_HOSTS 65536
 int nbos_place_batch_sequential(const nbos_snapshot *snap, const int32_t *requests,
                                 int64_t batch_per_snapshot, int32_t *out_hosts, int32_t *out_found,
                                 int32_t *out_subscribed, void *cuda_stream);

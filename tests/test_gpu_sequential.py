@@ -78,12 +78,34 @@ def test_cluster_fills_up(nb):
     assert (ref[1][0, :50] == 3).all() and (ref[1][0, -50:] < 3).all()
     cap = 32                                                    # raw limit 4 on 8 GPUs
     assert ref[2].max() <= cap
-    # the largest table the entry point takes
+    # the largest table one block takes
     check(nb, W.uniform_cluster(8192, 300, seed=10), what="8192 hosts")
     w = W.uniform_cluster(5000, 200, seed=11)
     w.requests[0, 3] = [-1, 0, 0, 0]
     w.requests[0, 4] = [0, 0, 0, 0]
     check(nb, w, what="5000 hosts, odd requests")
+
+
+@pytest.mark.parametrize("flags", [0, 2, 3], ids=["key32", "key64", "idle+key64"])
+def test_tables_spread_over_a_block_cluster(nb, flags):
+    """More than 8,192 hosts: 2, 4 or 8 blocks of a cluster share the table, ragged last block,
+    winners in different blocks and in the same block, several snapshots, odd requests."""
+    for hosts, batch, seed in ((8193, 120, 51), (20000, 150, 52), (40000, 60, 53), (65536, 40, 54)):
+        w = W.uniform_cluster(hosts, batch, seed=seed)
+        w.requests[0, 5] = [-1, 0, 0, 0]
+        w.requests[0, 6] = [0, 0, 0, 0]
+        check(nb, w, key_order=flags & 1, flags=flags, what=f"{hosts} hosts, flags {flags}")
+    w = W.mixed_gpu_cluster(12000, 200, seed=55)
+    check(nb, w, key_order=flags & 1, flags=flags, what="12000 mixed hosts")
+
+
+def test_cluster_form_fills_up_and_batches_snapshots(nb):
+    """Tight state on a large table: the best hosts sit in one block's run until they fill up and
+    the choice moves to the next; three snapshots run as three clusters."""
+    w = W.uniform_cluster(10000, 2500, seed=56, raw_limit="4")
+    ref = check(nb, w, what="10000 hosts, loose limit")
+    assert (ref[1] == 3).any()
+    check(nb, W.what_if_sweep(3, 9000, 100), what="three snapshots of 9000 hosts")
 
 
 def test_argument_errors(nb):
@@ -96,7 +118,7 @@ def test_argument_errors(nb):
         nb.nbos_place_batch_sequential(snap, req, out)
     assert e.value.status == nb.NBOS_ERR_INVALID_ARG
     nb.nbos_snapshot_destroy(snap)
-    big = W.uniform_cluster(8193, 8, seed=1)
+    big = W.uniform_cluster(65537, 8, seed=1)
     snap = nb.snapshot_from_workload(big, flags=nb.NBOS_ROOM_FOR_COMMITS)
     with pytest.raises(nb.NbosError) as e:
         nb.nbos_place_batch_sequential(snap, torch.from_numpy(big.requests).cuda(),
