@@ -3,6 +3,8 @@
 // scheduler designates (default policy order of Section 3.4.1 among those that can run).
 // One thread per kernel: a 128-bit request load, three host ids, three gathers from a packed
 // host table in shared memory, two 32-bit results. HBM-bound: 36 bytes per kernel.
+#include <limits.h>
+
 #include "nbos_internal.h"
 #include "nbos_ptx.cuh"
 
@@ -21,16 +23,17 @@ namespace {
 constexpr int kMemBits = 26, kIdleShift = 27, kIdleBits = 4, kVramBits = 11, kCpuShift = 12, kCpuBits = 19;
 constexpr unsigned int kGuardsX = (1u << kMemBits) | (1u << 31);
 constexpr unsigned int kGuardsY = (1u << kVramBits) | (1u << 31);
-// Order among runnable replicas with the same number of idle GPUs (Section 3.4.1): S / (G R)
-// ascending, R cancels; for 1 <= G <= 8 the integer S * (840 / G) orders the ratios exactly.
-constexpr int kRatioLcm = 840;
+// Order among runnable replicas (Section 3.4.1) as one 32-bit key per host, smaller first: 14 - idle
+// GPUs in the top four bits, below it S / (G R) as the integer S * (840 / G) -- R cancels, and for
+// 1 <= G <= 8 that integer orders the ratios exactly. Equal keys: the lower host index.
+constexpr int kRatioLcm = 840, kRatioBits = 28;
 constexpr int kPackBlock = 256;
 
 struct ExecArgs {
     const int4 *fit;        // [H] (idle GPUs or -1 if the host has none, vram_gb, millicpus, mem_mb)
     const int2 *rank;       // [H] (G, S): what the order among runnable replicas needs
     const uint2 *rec;       // [H + 1] packed form (above)
-    const unsigned int *ratio;  // [H + 1] S * (840 / G)
+    const unsigned int *ratio;  // [H + 1] designation key (above)
     const int *wide;        // [ceil(H / kPackBlock)] non-zero: some host of that block does not fit the packed form
     const int4 *requests;
     const int32_t *replica_hosts;
@@ -59,11 +62,12 @@ __global__ void __launch_bounds__(kPackBlock) pack_state_kernel(const int32_t *G
             rank[h] = make_int2(g, s);
             if ((f.x | f.y | f.z | f.w) >= 0) {   // otherwise the host runs nothing: GPU field 0
                 too_wide = f.x + 1 >= (1 << kIdleBits) || f.y >= (1 << kVramBits) || f.z >= (1 << kCpuBits) ||
-                           f.w >= (1 << kMemBits) || g > 8 || s < 0 || s >= (1 << 22);
+                           f.w >= (1 << kMemBits) || g > 8 || s < 0 ||
+                           (long long)s * (kRatioLcm / g) >= (1ll << kRatioBits);
                 if (!too_wide) {
                     r.x |= (unsigned int)f.w | ((unsigned int)(f.x + 1) << kIdleShift);
                     r.y |= (unsigned int)f.y | ((unsigned int)f.z << kCpuShift);
-                    q = (unsigned int)s * (unsigned int)(kRatioLcm / g);
+                    q = ((unsigned int)((1 << kIdleBits) - 2 - f.x) << kRatioBits) | ((unsigned int)s * (unsigned int)(kRatioLcm / g));
                 }
             }
         }
@@ -128,33 +132,21 @@ __device__ __forceinline__ void decide_packed(const uint2 *rec, const unsigned i
     // every host. (A GPU ask of 15 or more cannot be met by a host that fits the packed form.)
     const unsigned int qx = min((unsigned int)r.w, 1u << kMemBits) + ((min((unsigned int)r.x, (1u << kIdleBits) - 1u) + 1u) << kIdleShift);
     const unsigned int qy = min((unsigned int)r.y, 1u << kVramBits) + (min((unsigned int)r.z, 1u << kCpuBits) << kCpuShift);
-    unsigned int idle1[3];
+    unsigned int key[3];
     mask = 0;
 #pragma unroll
     for (int slot = 0; slot < 3; ++slot) {
-        const uint2 w = rec[min((unsigned int)h[slot], (unsigned int)H)];
+        const unsigned int idx = min((unsigned int)h[slot], (unsigned int)H);
+        const uint2 w = rec[idx];
+        const unsigned int dk = ratio[idx];
         const unsigned int lost = (~(w.x - qx) & kGuardsX) | (~(w.y - qy) & kGuardsY);
-        idle1[slot] = lost == 0u ? (w.x >> kIdleShift) & ((1u << kIdleBits) - 1u) : 0u;   // >= 1 when runnable
+        key[slot] = lost == 0u ? dk : 0xFFFFFFFFu;   // designation keys are below 15 << 28
         mask |= (lost == 0u ? 1 : 0) << slot;
     }
-    best = -1;
-    if (mask != 0) {
-        const unsigned int top = max(max(idle1[0], idle1[1]), idle1[2]);
-        const int first = (idle1[0] == top ? 1 : 0) | (idle1[1] == top ? 2 : 0) | (idle1[2] == top ? 4 : 0);
-        if ((first & (first - 1)) == 0) {
-            best = first == 1 ? h[0] : first == 2 ? h[1] : h[2];   // one replica has the most idle GPUs
-        } else {
-            // several with the same idle GPUs: lowest S / (G R), then lowest host index
-            unsigned long long key = ~0ull;
-#pragma unroll
-            for (int slot = 0; slot < 3; ++slot)
-                if ((first >> slot) & 1) {
-                    const unsigned long long k = ((unsigned long long)ratio[h[slot]] << 32) | (unsigned int)h[slot];
-                    key = k < key ? k : key;
-                }
-            best = (int)(unsigned int)key;
-        }
-    }
+    // smallest key, then smallest host index among those that have it (runnable slots hold valid indices)
+    const unsigned int m = min(min(key[0], key[1]), key[2]);
+    const int c0 = key[0] == m ? h[0] : INT_MAX, c1 = key[1] == m ? h[1] : INT_MAX, c2 = key[2] == m ? h[2] : INT_MAX;
+    best = mask != 0 ? min(min(c0, c1), c2) : -1;
 }
 
 // One kernel per thread and iteration. SMEM = true: the packed tables are first copied into
@@ -294,32 +286,37 @@ __global__ void __launch_bounds__(kRingThreads + 32, 2) select_executors_ring_ke
     asm volatile("bar.sync 1, %0;" ::"n"(kRingThreads) : "memory");
 
     bool ring_ok = true;
-    uint32_t i = 0;
-    for (long long t = blockIdx.x; t < full_tiles; t += gridDim.x, ++i) {
-        const uint32_t s = i % kRingStages, parity = (i / kRingStages) & 1u;
-        const long long k = t * kRingTile + tid;
-        int4 r;
-        int h[3];
-        // the whole warp takes the same path
-        if (ring_ok) ring_ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar + 8u * s, parity, abort_flag));
-        if (ring_ok) {
-            const unsigned char *stage = ring + (size_t)s * kRingStageBytes;
-            r = reinterpret_cast<const int4 *>(stage)[tid];
-            const int *ids = reinterpret_cast<const int *>(stage + kRingTile * 16u) + 3 * tid;
-            h[0] = ids[0];
-            h[1] = ids[1];
-            h[2] = ids[2];
-            __syncwarp();
-            if ((tid & 31) == 0) mbar_arrive(empty_bar + 8u * s);
-        } else {
-            r = __ldg(a.requests + k);
+    uint32_t parity = 0u;
+    const uint32_t tiles = (uint32_t)full_tiles;   // n_kernels <= 2^40: at most 2^31 tiles
+    for (uint32_t t0 = blockIdx.x; t0 < tiles; t0 += kRingStages * gridDim.x, parity ^= 1u) {
 #pragma unroll
-            for (int slot = 0; slot < 3; ++slot) h[slot] = __ldg(a.replica_hosts + 3 * k + slot);
+        for (int s = 0; s < kRingStages; ++s) {
+            const uint32_t t = t0 + (uint32_t)s * gridDim.x;
+            if (t >= tiles) break;
+            const long long k = (long long)t * kRingTile + tid;
+            int4 r;
+            int h[3];
+            // the whole warp takes the same path
+            if (ring_ok) ring_ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar + 8u * s, parity, abort_flag));
+            if (ring_ok) {
+                const unsigned char *stage = ring + (size_t)s * kRingStageBytes;
+                r = reinterpret_cast<const int4 *>(stage)[tid];
+                const int *ids = reinterpret_cast<const int *>(stage + kRingTile * 16u) + 3 * tid;
+                h[0] = ids[0];
+                h[1] = ids[1];
+                h[2] = ids[2];
+                __syncwarp();
+                if ((tid & 31) == 0) mbar_arrive(empty_bar + 8u * s);
+            } else {
+                r = __ldg(a.requests + k);
+#pragma unroll
+                for (int slot = 0; slot < 3; ++slot) h[slot] = __ldg(a.replica_hosts + 3 * k + slot);
+            }
+            int best, mask;
+            decide_packed(s_rec, s_ratio, a.H, r, h, best, mask);
+            a.out_executor[k] = best;
+            a.out_can_run[k] = mask;
         }
-        int best, mask;
-        decide_packed(s_rec, s_ratio, a.H, r, h, best, mask);
-        a.out_executor[k] = best;
-        a.out_can_run[k] = mask;
     }
     // what did not go through the ring: the partial last tile, or everything when the cluster
     // state needs the general form
