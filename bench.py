@@ -641,7 +641,8 @@ def run_ours(args):
 
         # sequential placement with commits: serial over requests, parallel over hosts / snapshots
         for label, ww in (("sequential_cfg4_shape", W.make_config(4)),
-                          ("sequential_one_snapshot_4096_hosts", W.make_config(3, batch=65_536))):
+                          ("sequential_one_snapshot_4096_hosts", W.make_config(3, batch=65_536)),
+                          ("sequential_one_snapshot_32768_hosts_block_cluster", W.uniform_cluster(32_768, 4096, seed=1))):
             sn = nb.snapshot_from_workload(ww, device=dev, flags=nb.NBOS_ROOM_FOR_COMMITS)
             rq = torch.from_numpy(ww.requests).to(dev)
             oh = torch.empty((ww.n_snapshots, ww.batch, 3), dtype=torch.int32, device=dev)

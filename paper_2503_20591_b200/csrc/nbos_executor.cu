@@ -149,32 +149,17 @@ __device__ __forceinline__ void decide_packed(const uint2 *rec, const unsigned i
     best = mask != 0 ? min(min(c0, c1), c2) : -1;
 }
 
-// One kernel per thread and iteration. SMEM = true: the packed tables are first copied into
-// shared memory (scattered reads from shared memory are several times cheaper than from L1, whose
-// tag stage handles one cache line per cycle; 8-byte records meet about half the bank conflicts
-// of 16-byte ones); SMEM = false: gathers go to global memory (tables too large for shared memory,
-// or too few kernels to pay for the copy). A cluster state that the packed form cannot hold
-// (flagged by the packing kernel) takes the general form with gathers from global memory.
-template <bool SMEM>
-__global__ void __launch_bounds__(512, SMEM ? 3 : 2) select_executors_kernel(const ExecArgs a)
+// One kernel per thread and iteration, gathers from the packed tables in global memory (they stay
+// in L1 / L2). Used for small batches, for tables too large for shared memory, and for host-id
+// arrays that are not 16-byte aligned; large batches take the ring form below. A cluster state
+// that the packed form cannot hold (flagged by the packing kernel) takes the general form.
+__global__ void __launch_bounds__(512, 2) select_executors_kernel(const ExecArgs a)
 {
-    extern __shared__ __align__(16) unsigned char exec_smem[];
     const uint2 *rec = a.rec;
     const unsigned int *ratio = a.ratio;
     int wide = 0;
     for (int i = threadIdx.x; i * kPackBlock < a.H; i += blockDim.x) wide |= a.wide[i];
     wide = __syncthreads_or(wide);
-    if (SMEM && !wide) {
-        uint2 *s_rec = reinterpret_cast<uint2 *>(exec_smem);
-        unsigned int *s_ratio = reinterpret_cast<unsigned int *>(exec_smem + (size_t)(a.H + 1) * sizeof(uint2));
-        for (int i = threadIdx.x; i <= a.H; i += blockDim.x) {
-            s_rec[i] = a.rec[i];
-            s_ratio[i] = a.ratio[i];
-        }
-        __syncthreads();
-        rec = s_rec;
-        ratio = s_ratio;
-    }
     // the streams of the next iteration are requested before this iteration's records are
     // gathered, so that every thread always has a request and three host ids in flight
     const long long stride = (long long)gridDim.x * blockDim.x;
@@ -398,25 +383,19 @@ extern "C" int nbos_select_executors(const nbos_cluster_state *state, const int3
     if (e == cudaSuccess) {
         ExecArgs a{fit, rank, rec, ratio, wide, reinterpret_cast<const int4 *>(requests), replica_hosts,
                    out_executor, out_can_run, n_kernels, H};
-        const size_t table_bytes = (size_t)(H + 1) * (sizeof(uint2) + sizeof(unsigned int));
-        const bool use_smem = table_bytes <= 72 * 1024 && n_kernels >= (long long)sms * 2 * 8 * H;
-        const size_t ring_table = (table_bytes + 127) & ~(size_t)127;
-        const size_t ring_smem = ring_table + (size_t)kRingStages * kRingStageBytes + 2 * kRingStages * 8 + 16;
-        const bool use_ring = use_smem && ring_smem <= 110 * 1024 && aligned16(replica_hosts) &&
-                              n_kernels >= (long long)sms * 2 * kRingTile * 4;
+        // the ring form pays from about half a million kernels on (measured: never slower than
+        // the plain form from 2^20 kernels, 15 - 25 % faster at 2^22 and above)
+        const size_t table_bytes = ((size_t)(H + 1) * (sizeof(uint2) + sizeof(unsigned int)) + 127) & ~(size_t)127;
+        const size_t ring_smem = table_bytes + (size_t)kRingStages * kRingStageBytes + 2 * kRingStages * 8 + 16;
+        const bool use_ring = ring_smem <= 110 * 1024 && aligned16(replica_hosts) && n_kernels >= (1ll << 19);
         if (use_ring) {
             e = cudaFuncSetAttribute(select_executors_ring_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ring_smem);
             if (e == cudaSuccess)
-                select_executors_ring_kernel<<<sms * 2, kRingThreads + 32, ring_smem, stream>>>(a, (int)ring_table);
-        } else if (use_smem) {
-            e = cudaFuncSetAttribute(select_executors_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)table_bytes);
-            if (e == cudaSuccess)
-                select_executors_kernel<true><<<sms * 3, 512, table_bytes, stream>>>(a);
+                select_executors_ring_kernel<<<sms * 2, kRingThreads + 32, ring_smem, stream>>>(a, (int)table_bytes);
         } else {
             long long blocks = (n_kernels + 511) / 512;
             if (blocks > (long long)sms * 4) blocks = (long long)sms * 4;
-            select_executors_kernel<false><<<(unsigned int)blocks, 512, 0, stream>>>(a);
+            select_executors_kernel<<<(unsigned int)blocks, 512, 0, stream>>>(a);
         }
         e = cudaGetLastError();
     }

@@ -114,7 +114,7 @@ def edge_asks(rng, m, hosts):
 
 
 @pytest.mark.parametrize("hosts,m", [(7, 3000), (300, 40_000), (300, 1_000_003), (4096, 2_500_000), (4096, 10_000_002),
-                                     (4300, 11_000_000), (7000, 400_000), (40_000, 300_000)])
+                                     (4300, 11_000_000), (5000, 700_000), (7000, 400_000), (40_000, 300_000)])
 def test_ties_dead_hosts_and_edge_asks(nb, hosts, m):
     """Packed 8-byte host records, tables in shared memory (many kernels per host: inputs through
     the ring of bulk copies, whole tiles and a partial last one) and in global memory (few kernels,
@@ -126,6 +126,25 @@ def test_ties_dead_hosts_and_edge_asks(nb, hosts, m):
     assert (ref[0] >= 0).any() and (ref[0] < 0).any()
     several = np.array([bin(x).count("1") for x in ref[1][:5000]]) >= 2
     assert several.any()
+
+
+def test_host_ids_not_16_byte_aligned(nb):
+    """A large batch whose host-id array starts 12 bytes into an allocation: no bulk copies, plain loads."""
+    import torch
+    rng = np.random.default_rng(77)
+    hosts, m = 1000, 800_000
+    state = crowded_state(rng, hosts)
+    req, rep = edge_asks(rng, m + 1, hosts)
+    dev = [torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).cuda() for a in state]
+    rep_dev = torch.from_numpy(rep).cuda()[1:]
+    assert rep_dev.data_ptr() % 16 == 12
+    ex = torch.full((m,), -9, dtype=torch.int32, device="cuda")
+    mask = torch.full((m,), -9, dtype=torch.int32, device="cuda")
+    nb.nbos_select_executors(*dev, torch.from_numpy(req[1:]).cuda(), rep_dev, ex, mask)
+    torch.cuda.synchronize()
+    ref = oracle.select_executors(*[np.ascontiguousarray(a, dtype=np.int32) for a in state], req[1:], rep[1:])
+    np.testing.assert_array_equal(mask.cpu().numpy(), ref[1])
+    np.testing.assert_array_equal(ex.cpu().numpy(), ref[0])
 
 
 @pytest.mark.parametrize("what", ["gpus", "memory", "cpu", "vram", "subscribed", "idle", "last_host_only"])
