@@ -522,13 +522,14 @@ def run_ours(args):
                        f"{sm_mhz:.0f} MHz sampled during the timed region; probe_both_gops is this "
                        "peak measured in the same process, probe_alu_gops / probe_imad_gops each pipe alone",
         "pair_evaluation": ("ranked form: every (request, host) pair is tested against its own request -- the four "
-                            "capacities and the host's rank against the request's current third best -- by one 64-bit "
-                            "subtraction and one logic operation; no request is ever switched off"
+                            "capacities and the host's rank against the request's current third best -- by one packed 32-bit "
+                            "subtraction and one logic operation (a second, finer level and the exact test only for "
+                            "the few pairs that pass); no request is ever switched off"
                             if (info.ranked and not args.pair_mode) else f"pair_mode {args.pair_mode}"),
         "note": "achieved counts the 6 algorithmic operations of a pair (4 capacity compares, key multiply-add, "
-                "compare with the third best). The kernel executes about 3.5 instructions per pair: the five "
-                "compares share one packed subtraction and its guard test, and the key is the host's "
-                "precomputed rank. So frac can exceed 1; issue_slot_frac is the executed-instruction view "
+                "compare with the third best). The kernel executes fewer instructions per pair than that "
+                "(warp_instructions_per_32_pairs): the five compares share one packed subtraction and its "
+                "guard test, and the key is the host's precomputed rank. So frac can exceed 1; issue_slot_frac is the executed-instruction view "
                 "of the same launch (warp instructions issued / issue slots)",
         "ops_per_pair": ALGORITHMIC_OPS_PER_PAIR, "kernel_ms": kern_ms,
         "kernel_ms_min": min(kern_ms_all), "kernel_launches_timed": len(kern_ms_all),

@@ -317,10 +317,12 @@ int nbos_place_batch_noalloc(const nbos_snapshot *snap, const int32_t *requests,
  *   state          DEVICE arrays [n_hosts] int32 of one cluster snapshot (not validated; a host
  *                  index outside 0..n_hosts-1 in replica_hosts, e.g. -1, means "no such replica")
  *   requests       DEVICE [n_kernels * 4] int32, 16-byte aligned: GPUs, VRAM GB, millicpus, MB
- *   replica_hosts  DEVICE [n_kernels * 3] int32
+ *   replica_hosts  DEVICE [n_kernels * 3] int32 (any 4-byte alignment; when it is 16-byte aligned,
+ *                  batches of 2^19 kernels and more are streamed through bulk asynchronous copies)
  *   out_executor   DEVICE [n_kernels] int32: host index of the designated executor, -1 = all yield
  *   out_can_run    DEVICE [n_kernels] int32: bit k set = the replica in slot k can run now
- * Asynchronous on `cuda_stream`. Errors: INVALID_ARG, CUDA, UNSUPPORTED_DEVICE.
+ * Asynchronous on `cuda_stream`; a per-call temporary of 36 bytes per host comes from the
+ * library's stream-ordered pool. Errors: INVALID_ARG, NO_MEMORY, CUDA, UNSUPPORTED_DEVICE.
  */
 typedef struct nbos_cluster_state {
     int32_t n_hosts;
