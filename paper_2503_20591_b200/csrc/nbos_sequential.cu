@@ -4,14 +4,14 @@
 // parallelism is over hosts (all hosts of the snapshot are evaluated for one request at a time)
 // and over snapshots (one thread block each).
 //
-// One block of 1,024 threads owns a snapshot. Thread t owns hosts t, t + 1024, ...: the fields a
-// commit changes (room under the SR limit, key intercept A) live in registers, the static ones in
-// shared memory. Per request: every thread ranks its own hosts, each warp extracts its three
-// smallest keys with three warp-wide integer minimum reductions (keys are unique, the lane that
-// held the minimum pops it), warp 0 does the same over the warps' triples, writes the result,
-// and the owners of the three winning hosts update them. Two block barriers per request.
-// (512 threads with twice the hosts each were measured slower: the per-thread chain of
-// best-three insertions is the critical path, not the per-warp reduction cost.)
+// One block of T = 256, 512 or 1,024 threads owns a snapshot (about four hosts per thread; up to
+// eight at 8,192 hosts). Thread t owns hosts t, t + T, ...: the fields a commit changes (room under
+// the SR limit, key intercept A) live in registers, the static ones in shared memory. Per
+// request: every thread ranks its own hosts, each warp extracts its three smallest keys with
+// three warp-wide integer minimum reductions (keys are unique, the lane that held the minimum
+// pops it) and writes them to shared memory; behind one block barrier every warp does the same
+// over the warps' triples for itself, thread 0 writes the result, and the owners of the three
+// winning hosts update them. One block barrier per request.
 //
 // Tables beyond 8,192 hosts (what one block's registers and shared memory hold) are spread over a
 // thread-block cluster of 2, 4 or 8 blocks, each owning a contiguous run of the hosts. Per request
@@ -81,18 +81,21 @@ __device__ __forceinline__ void warp_best3(KeyT k1, KeyT k2, KeyT k3, KeyT &w1, 
     w1 = w[0]; w2 = w[1]; w3 = w[2];
 }
 
-// HPT = hosts per thread (1..8). Static per-host fields in shared memory: (vram, cpu, mem, g_cap) as int4
-// and B; dynamic in registers: room = cap - S, A, and the GPUs added so far.
-template <typename KeyT, int HPT>
-__global__ void __launch_bounds__(kSeqThreads, 1) place_sequential_kernel(const SeqParams p)
+// T threads, HPT hosts per thread (1..8). Static per-host fields in shared memory: (vram, cpu, mem,
+// g_cap) as int4 and B; dynamic in registers: room = cap - S, A, and the GPUs added so far.
+// One block barrier per request: every warp writes its best three, and behind the barrier every
+// warp reduces the T / 32 triples for itself (the buffer alternates with the request's parity, so
+// a warp that runs ahead never overwrites what a slower one still reads).
+template <typename KeyT, int HPT, int T>
+__global__ void __launch_bounds__(T) place_sequential_kernel(const SeqParams p)
 {
     using Pair = typename SeqKey<KeyT>::Pair;
     constexpr KeyT kInf = SeqKey<KeyT>::kInf;
+    constexpr int W = T / 32;
     extern __shared__ __align__(16) unsigned char seq_smem[];
-    int4 *s_cap = reinterpret_cast<int4 *>(seq_smem);                                        // [HPT*1024]
-    KeyT *s_B = reinterpret_cast<KeyT *>(seq_smem + (size_t)HPT * kSeqThreads * sizeof(int4));  // [HPT*1024]
-    __shared__ KeyT s_warp[kSeqWarps][3];
-    __shared__ KeyT s_best[3];
+    int4 *s_cap = reinterpret_cast<int4 *>(seq_smem);                              // [HPT * T]
+    KeyT *s_B = reinterpret_cast<KeyT *>(seq_smem + (size_t)HPT * T * sizeof(int4));  // [HPT * T]
+    __shared__ KeyT s_warp[2][W][3];
 
     const int n = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -102,7 +105,7 @@ __global__ void __launch_bounds__(kSeqThreads, 1) place_sequential_kernel(const 
     KeyT A[HPT];
 #pragma unroll
     for (int u = 0; u < HPT; ++u) {
-        const int h = tid + u * kSeqThreads;
+        const int h = tid + u * T;
         int4 cap = make_int4(0, 0, 0, -1);
         KeyT b = 0;
         room[u] = -1;
@@ -131,49 +134,47 @@ __global__ void __launch_bounds__(kSeqThreads, 1) place_sequential_kernel(const 
     for (long long r = 0; r < p.B; ++r) {
         const int4 q = next;
         if (r + 1 < p.B) next = __ldg(req + r + 1);
+        const int par = (int)(r & 1);
         const bool sane = (q.x | q.y | q.z | q.w) >= 0;
         KeyT k1 = kInf, k2 = kInf, k3 = kInf;
         if (sane) {
 #pragma unroll
             for (int u = 0; u < HPT; ++u) {
-                const int h = tid + u * kSeqThreads;
+                const int h = tid + u * T;
                 const int4 cap = s_cap[h];
                 const bool ok = q.x <= gmax_now[u] && q.y <= cap.x && q.z <= cap.y && q.w <= cap.z;
                 const KeyT key = ok ? (KeyT)(A[u] + (KeyT)(unsigned int)q.x * s_B[h]) : kInf;
                 insert3(k1, k2, k3, key);
             }
         }
-        KeyT w1, w2, w3;
-        warp_best3(k1, k2, k3, w1, w2, w3);
-        if (lane == 0) {
-            s_warp[warp][0] = w1;
-            s_warp[warp][1] = w2;
-            s_warp[warp][2] = w3;
-        }
-        __syncthreads();
-        if (warp == 0) {
-            KeyT b1, b2, b3;
-            const bool has = lane < kSeqWarps;
-            warp_best3(has ? s_warp[lane][0] : kInf, has ? s_warp[lane][1] : kInf, has ? s_warp[lane][2] : kInf, b1, b2, b3);
+        KeyT b1, b2, b3;
+        warp_best3(k1, k2, k3, b1, b2, b3);
+        if (W > 1) {
             if (lane == 0) {
-                s_best[0] = b1;
-                s_best[1] = b2;
-                s_best[2] = b3;
-                const long long o = (long long)n * p.B + r;
-                p.out_hosts[o * 3 + 0] = b1 == kInf ? -1 : (int)((unsigned int)b1 & p.id_mask);
-                p.out_hosts[o * 3 + 1] = b2 == kInf ? -1 : (int)((unsigned int)b2 & p.id_mask);
-                p.out_hosts[o * 3 + 2] = b3 == kInf ? -1 : (int)((unsigned int)b3 & p.id_mask);
-                if (p.out_found) p.out_found[o] = (b1 != kInf) + (b2 != kInf) + (b3 != kInf);
+                s_warp[par][warp][0] = b1;
+                s_warp[par][warp][1] = b2;
+                s_warp[par][warp][2] = b3;
             }
+            __syncthreads();
+            const bool has = lane < W;
+            warp_best3(has ? s_warp[par][has ? lane : 0][0] : kInf, has ? s_warp[par][has ? lane : 0][1] : kInf,
+                       has ? s_warp[par][has ? lane : 0][2] : kInf, b1, b2, b3);
         }
-        __syncthreads();
+        if (tid == 0) {
+            const long long o = (long long)n * p.B + r;
+            p.out_hosts[o * 3 + 0] = b1 == kInf ? -1 : (int)((unsigned int)b1 & p.id_mask);
+            p.out_hosts[o * 3 + 1] = b2 == kInf ? -1 : (int)((unsigned int)b2 & p.id_mask);
+            p.out_hosts[o * 3 + 2] = b3 == kInf ? -1 : (int)((unsigned int)b3 & p.id_mask);
+            if (p.out_found) p.out_found[o] = (b1 != kInf) + (b2 != kInf) + (b3 != kInf);
+        }
         // commit: only a kernel that got all three replicas is created
-        if (s_best[2] != kInf && q.x > 0) {
+        if (b3 != kInf && q.x > 0) {
+            const KeyT best[3] = {b1, b2, b3};
 #pragma unroll
             for (int i = 0; i < 3; ++i) {
-                const int h = (int)((unsigned int)s_best[i] & p.id_mask);
-                if ((h & (kSeqThreads - 1)) == tid) {
-                    const int u0 = h / kSeqThreads;
+                const int h = (int)((unsigned int)best[i] & p.id_mask);
+                if ((h & (T - 1)) == tid) {
+                    const int u0 = h / T;
 #pragma unroll
                     for (int u = 0; u < HPT; ++u)
                         if (u == u0) {
@@ -185,13 +186,11 @@ __global__ void __launch_bounds__(kSeqThreads, 1) place_sequential_kernel(const 
                 }
             }
         }
-        // s_best is rewritten only after the next request's first barrier, which every thread
-        // reaches after having read it here
     }
     if (p.out_subscribed) {
 #pragma unroll
         for (int u = 0; u < HPT; ++u) {
-            const int h = tid + u * kSeqThreads;
+            const int h = tid + u * T;
             if (h < p.H) p.out_subscribed[(size_t)n * p.H + h] = p.seq[row + h].z + added[u];
         }
     }
@@ -369,18 +368,28 @@ int launch_seq_cluster(const SeqParams &p, int N, int C, cudaStream_t stream)
     return NBOS_OK;
 }
 
-template <typename KeyT>
-int launch_seq(const SeqParams &p, int N, int hpt, cudaStream_t stream)
+template <typename KeyT, int T>
+int launch_seq_t(const SeqParams &p, int N, int hpt, cudaStream_t stream)
 {
-    const size_t smem = (size_t)hpt * kSeqThreads * (sizeof(int4) + sizeof(KeyT));
-    void (*fn)(const SeqParams) = hpt == 1 ? place_sequential_kernel<KeyT, 1>
-                                  : hpt == 2 ? place_sequential_kernel<KeyT, 2>
-                                  : hpt == 4 ? place_sequential_kernel<KeyT, 4>
-                                             : place_sequential_kernel<KeyT, 8>;
+    const size_t smem = (size_t)hpt * T * (sizeof(int4) + sizeof(KeyT));
+    void (*fn)(const SeqParams) = hpt == 1 ? place_sequential_kernel<KeyT, 1, T>
+                                  : hpt == 2 ? place_sequential_kernel<KeyT, 2, T>
+                                  : hpt == 4 ? place_sequential_kernel<KeyT, 4, T>
+                                             : place_sequential_kernel<KeyT, 8, T>;
     NBOS_CUDA_TRY(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    fn<<<N, kSeqThreads, smem, stream>>>(p);
+    fn<<<N, T, smem, stream>>>(p);
     NBOS_CUDA_TRY(cudaGetLastError());
     return NBOS_OK;
+}
+
+template <typename KeyT>
+int launch_seq(const SeqParams &p, int N, int threads, int hpt, cudaStream_t stream)
+{
+    switch (threads) {
+    case 256: return launch_seq_t<KeyT, 256>(p, N, hpt, stream);
+    case 512: return launch_seq_t<KeyT, 512>(p, N, hpt, stream);
+    default: return launch_seq_t<KeyT, 1024>(p, N, hpt, stream);
+    }
 }
 
 }  // namespace
@@ -409,10 +418,14 @@ int launch_place_sequential(const nbos_snapshot *s, const int32_t *d_requests, i
         return s->key.key_bits == 64 ? launch_seq_cluster<unsigned long long>(p, s->N, C, stream)
                                      : launch_seq_cluster<unsigned int>(p, s->N, C, stream);
     }
+    // about four hosts per thread is fastest (measured at 256 to 8,192 hosts, one snapshot and 256):
+    // fewer warps make the two reductions and the barrier cheaper, more hosts per thread lengthen
+    // the evaluation; small blocks also let several snapshots share an SM
+    const int threads = s->Hpad <= 1024 ? 256 : s->Hpad <= 2048 ? 512 : 1024;
     int hpt = 1;
-    while (hpt * kSeqThreads < s->Hpad) hpt <<= 1;
-    return s->key.key_bits == 64 ? launch_seq<unsigned long long>(p, s->N, hpt, stream)
-                                 : launch_seq<unsigned int>(p, s->N, hpt, stream);
+    while (hpt * threads < s->Hpad) hpt <<= 1;
+    return s->key.key_bits == 64 ? launch_seq<unsigned long long>(p, s->N, threads, hpt, stream)
+                                 : launch_seq<unsigned int>(p, s->N, threads, hpt, stream);
 }
 
 }  // namespace nbos
