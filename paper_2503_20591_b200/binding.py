@@ -31,6 +31,10 @@ NBOS_FORCE_KEY64 = 2
 NBOS_LIMIT_CLUSTER_SR = 4
 NBOS_ROOM_FOR_COMMITS = 8
 
+NBOS_MAX_HOSTS = 1 << 20
+NBOS_MAX_REPLICAS = 1024
+NBOS_SEQUENTIAL_MAX_HOSTS = 65536
+
 NBOS_PROBE_MIX_ALU = 0
 NBOS_PROBE_MIX_IMAD = 1
 NBOS_PROBE_MIX_BOTH = 2

@@ -34,6 +34,22 @@ def test_every_declared_symbol_is_exported(lib):
     assert sorted(binding.EXPORTED_SYMBOLS) == names
 
 
+def test_binding_constants_match_the_header():
+    """Every NBOS_* constant of the binding has the value include/nbos.h defines."""
+    import re
+    text = open(os.path.join(ROOT, "include", "nbos.h")).read() + open(os.path.join(ROOT, "include", "nbos_probe.h")).read()
+    defines = {m.group(1): m.group(2).strip() for m in re.finditer(r"#define\s+(NBOS_[A-Z0-9_]+)\s+([^/\n]+)", text)}
+    enums = {m.group(1): m.group(2).strip() for m in re.finditer(r"\b(NBOS_[A-Z0-9_]+)\s*=\s*(-?\d+)", text)}
+    known = {**enums, **defines}
+    checked = 0
+    for name in dir(binding):
+        if name.startswith("NBOS_") and isinstance(getattr(binding, name), int) and name in known:
+            assert getattr(binding, name) == eval(known[name].strip("()").replace("u", "")), name
+            checked += 1
+    assert checked >= 12
+    assert binding.NBOS_MAX_HOSTS == 1 << 20 and binding.NBOS_SEQUENTIAL_MAX_HOSTS == 65536
+
+
 def test_strerror(lib):
     assert binding.nbos_strerror(0) == "ok"
     for code in range(-6, 0):

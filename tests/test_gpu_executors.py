@@ -114,7 +114,7 @@ def edge_asks(rng, m, hosts):
 
 
 @pytest.mark.parametrize("hosts,m", [(7, 3000), (300, 40_000), (300, 1_000_003), (4096, 2_500_000), (4096, 10_000_002),
-                                     (4300, 11_000_000), (5000, 700_000), (7000, 400_000), (40_000, 300_000)])
+                                     (4300, 11_000_000), (5000, 700_000), (7000, 400_000), (40_000, 300_000), (1 << 20, 600_000)])
 def test_ties_dead_hosts_and_edge_asks(nb, hosts, m):
     """Packed 8-byte host records, tables in shared memory (many kernels per host: inputs through
     the ring of bulk copies, whole tiles and a partial last one) and in global memory (few kernels,

@@ -358,6 +358,27 @@ def test_large_tables(nb):
         assert_same(got, ref, f"70000 hosts {shape}")
 
 
+def test_maximum_table_sizes(nb):
+    """The largest table stored in key order (65,536 hosts: the position count is quadratic) and
+    the largest table the library takes (2^20 hosts, host order, 64-bit keys)."""
+    w = W.uniform_cluster(65_536, 96, seed=81)
+    s = nb.snapshot_from_workload(w)
+    assert s.info().presorted == 1
+    nb.nbos_snapshot_destroy(s)
+    got, ref = both(nb, w)
+    assert_same(got, ref, "65,536 hosts")
+    w = W.mixed_gpu_cluster(65_536, 40, seed=82)
+    got, ref = both(nb, w)
+    assert_same(got, ref, "65,536 mixed hosts")
+    w = W.uniform_cluster(nb.NBOS_MAX_HOSTS, 24, seed=83)
+    got, ref = both(nb, w)
+    assert_same(got, ref, "2^20 hosts")
+    assert (ref[1] == 3).all()
+    w = W.mixed_gpu_cluster(nb.NBOS_MAX_HOSTS, 12, seed=84)
+    got, ref = both(nb, w, key_order=1)
+    assert_same(got, ref, "2^20 mixed hosts, SR first")
+
+
 def test_key_width_is_chosen_from_the_data(nb):
     w = W.make_config(1)
     s = nb.snapshot_from_workload(w)
