@@ -449,46 +449,76 @@ def run_ours(args):
     if not args.no_e2e:
         h_state = [torch.from_numpy(getattr(w, k)).reshape(-1).pin_memory() for k in w.HOST_FIELDS]
         h_req = [torch.from_numpy(np.ascontiguousarray(b[:, lo:hi])).pin_memory() for b in batches[:2]]
-        h_out = torch.empty((w.n_snapshots, my_batch, 3), dtype=torch.int32).pin_memory()
-        h_found = torch.empty((w.n_snapshots, my_batch), dtype=torch.int32).pin_memory()
+        h_out = [torch.empty((w.n_snapshots, my_batch, 3), dtype=torch.int32).pin_memory() for _ in range(2)]
+        h_found = [torch.empty((w.n_snapshots, my_batch), dtype=torch.int32).pin_memory() for _ in range(2)]
 
         e2e_live = None if args.fresh_snapshot else nb.nbos_snapshot_create_host(
             w.n_snapshots, w.n_hosts, lim_num, lim_den, *h_state, replicas_R=w.replicas_R, stream=stream)
 
-        def e2e_step(i):
+        def e2e_step(i, blocking):
             if e2e_live is None:
                 snap = nb.nbos_snapshot_create_host(w.n_snapshots, w.n_hosts, lim_num, lim_den,
                                                     *h_state, replicas_R=w.replicas_R, stream=stream)
             else:
                 snap = e2e_live
                 nb.nbos_snapshot_update_host(snap, lim_num, lim_den, *h_state, stream=stream)
-            nb.nbos_place_batch_host(snap, h_req[i % 2], h_out, h_found, stream=stream)
+            place = nb.nbos_place_batch_host if (blocking or e2e_live is None) else nb.nbos_place_batch_host_async
+            place(snap, h_req[i % 2], h_out[i % 2], h_found[i % 2], stream=stream)
             if e2e_live is None:
                 nb.nbos_snapshot_destroy(snap)
 
         e2e_steps = max(3, min(args.steps, 50))
-        for i in range(3):
-            e2e_step(i)
-        sync_all()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e2e_rounds = []
-        while True:
-            a.record(stream)
-            for i in range(e2e_steps):
-                e2e_step(i)
-            b.record(stream)
+
+        def e2e_time(blocking):
+            for i in range(3):
+                e2e_step(i, blocking)
+            if not blocking and e2e_live is not None:
+                nb.nbos_place_batch_host_wait(e2e_live)
             sync_all()
-            e2e_rounds.append(max_over_ranks(a.elapsed_time(b)))
-            if sum(e2e_rounds) >= 0.5 * args.min_timed_ms or len(e2e_rounds) >= args.max_rounds:
-                break
-        e2e_ms = statistics.median(e2e_rounds) / e2e_steps
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            rounds = []
+            while True:
+                a.record(stream)
+                for i in range(e2e_steps):
+                    e2e_step(i, blocking)
+                if not blocking and e2e_live is not None:
+                    nb.nbos_place_batch_host_wait(e2e_live)    # the last results are in the host buffers
+                b.record(stream)
+                sync_all()
+                rounds.append(max_over_ranks(a.elapsed_time(b)))
+                if sum(rounds) >= 0.5 * args.min_timed_ms or len(rounds) >= args.max_rounds:
+                    break
+            return statistics.median(rounds) / e2e_steps, len(rounds)
+
+        blocking_ms, blocking_rounds = e2e_time(True)
+        e2e_ms, e2e_rounds = e2e_time(False)
+        # what the last two queued steps left in the host buffers against the device path on the same requests
+        same = True
+        chk = e2e_live if e2e_live is not None else nb.nbos_snapshot_create_host(
+            w.n_snapshots, w.n_hosts, lim_num, lim_den, *h_state, replicas_R=w.replicas_R, stream=stream)
+        for k in range(2):
+            d_req_k = h_req[k].to(dev)
+            d_out_k = torch.empty((w.n_snapshots, my_batch, 3), dtype=torch.int32, device=dev)
+            d_found_k = torch.empty((w.n_snapshots, my_batch), dtype=torch.int32, device=dev)
+            nb.nbos_place_batch(chk, d_req_k, d_out_k, d_found_k, stream=stream)
+            sync_all()
+            same = same and bool(torch.equal(d_out_k.cpu(), h_out[k])) and bool(torch.equal(d_found_k.cpu(), h_found[k]))
         h2d = w.n_snapshots * my_batch * 16 + 6 * 4 * w.n_snapshots * w.n_hosts + 8 * w.n_snapshots
         d2h = w.n_snapshots * my_batch * (12 + 4)
-        if e2e_live is not None:
-            nb.nbos_snapshot_destroy(e2e_live)
+        nb.nbos_snapshot_destroy(chk)
         e2e = {"value": decisions_all / (e2e_ms * 1e-3), "unit": "decisions/s",
-               "ms_per_step": e2e_ms, "steps": e2e_steps, "rounds": len(e2e_rounds),
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "host_memory": "pinned"}
+               "ms_per_step": e2e_ms, "steps": e2e_steps, "rounds": e2e_rounds,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "host_memory": "pinned",
+               "mode": ("every step = nbos_snapshot_update_host + nbos_place_batch_host_async from and to pinned host "
+                        "buffers (two request / result buffer sets in turn); steps are queued without waiting in "
+                        "between, so the copies in of one step run beside the kernels and copies out of the step "
+                        "before; the timed region ends after nbos_place_batch_host_wait, so all copies of all timed steps lie inside it"
+                        if e2e_live is not None else "fresh snapshot per step, blocking calls"),
+               "blocking_call": {"value": decisions_all / (blocking_ms * 1e-3), "ms_per_step": blocking_ms,
+                                 "rounds": blocking_rounds,
+                                 "note": "nbos_place_batch_host: returns with the results in the host buffers, "
+                                         "one step at a time (the latency of a step)"},
+               "output_identical_to_device_path": same}
 
     if rank != 0:
         if dist is not None:

@@ -251,15 +251,33 @@ int nbos_place_batch_ex(const nbos_snapshot *snap, const int32_t *requests,
 /*
  * Same operation with HOST buffers (pinned memory makes the copies asynchronous and faster, but
  * any host memory works). The batch is cut into up to 4 chunks whose host-to-device copy, kernel
- * and device-to-host copy overlap on three internal streams (created once per device; calls on
- * the same device take turns). The copies in start at once; the kernels wait for the work queued
- * on `cuda_stream` before the call (a snapshot update, say). Device staging is a buffer the library
- * keeps per device and grows when a larger batch comes. Returns after the results are in the host
- * buffers.
+ * and device-to-host copy overlap on three internal streams (copies in, kernels, copies out;
+ * created once per device, with two sets of device staging that successive calls take in turn and
+ * that grow when a larger batch comes). The copies in start as soon as staging is free; the
+ * kernels wait for the work queued on `cuda_stream` before the call (a snapshot update, say), and
+ * `cuda_stream` in turn waits for the kernels, so that a later update of the snapshot queued on it
+ * does not overtake them. Calls on the same device take their turns in the order they are made.
+ *   nbos_place_batch_host        returns after the results are in the host buffers.
+ *   nbos_place_batch_host_async  returns once the work is queued. Calls in a row overlap: the
+ *                                copies in of one run beside the kernels of the one before and
+ *                                the copies out of the one before that. The request and result
+ *                                buffers belong to the library until nbos_place_batch_host_wait
+ *                                (or a later nbos_place_batch_host on the same device) has
+ *                                returned. With pageable host memory the copies block the caller
+ *                                and nothing overlaps (still correct).
+ *   nbos_place_batch_host_wait   blocks until every host-buffer call made so far on the
+ *                                snapshot's device has delivered its results. Call it before
+ *                                destroying a snapshot that asynchronous calls still use.
+ * Errors: INVALID_ARG, NO_MEMORY, CUDA (after an error the internal streams are synchronised
+ * before the call returns).
  */
 int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_host,
                           int64_t batch_per_snapshot, int32_t *out_hosts_host,
                           int32_t *out_found_host, void *cuda_stream);
+int nbos_place_batch_host_async(const nbos_snapshot *snap, const int32_t *requests_host,
+                                int64_t batch_per_snapshot, int32_t *out_hosts_host,
+                                int32_t *out_found_host, void *cuda_stream);
+int nbos_place_batch_host_wait(const nbos_snapshot *snap);
 
 /*
  * Placement for callers that are not allowed to allocate device memory. (The paper has no

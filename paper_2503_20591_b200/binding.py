@@ -44,7 +44,8 @@ EXPORTED_SYMBOLS = (
     "nbos_snapshot_workspace_bytes", "nbos_snapshot_create", "nbos_snapshot_create_host",
     "nbos_snapshot_update", "nbos_snapshot_update_host",
     "nbos_snapshot_destroy", "nbos_snapshot_get_info", "nbos_place_batch", "nbos_place_batch_ex",
-    "nbos_place_batch_host", "nbos_place_batch_noalloc", "nbos_select_executors",
+    "nbos_place_batch_host", "nbos_place_batch_host_async", "nbos_place_batch_host_wait",
+    "nbos_place_batch_noalloc", "nbos_select_executors",
     "nbos_cluster_sums", "nbos_scale_out_deficit", "nbos_place_batch_sequential",
     "nbos_snapshot_status", "nbos_strerror", "nbos_last_error_detail",
     "nbos_probe_int32_issue", "nbos_probe_wait_timeout", "nbos_probe_wait_timeout_on_snapshot",
@@ -128,6 +129,8 @@ def load_library() -> ctypes.CDLL:
     lib.nbos_place_batch.argtypes = [vp, vp, i64, vp, vp, vp]
     lib.nbos_place_batch_ex.argtypes = [vp, vp, i64, vp, vp, vp, P(nbos_launch_config)]
     lib.nbos_place_batch_host.argtypes = [vp, vp, i64, vp, vp, vp]
+    lib.nbos_place_batch_host_async.argtypes = [vp, vp, i64, vp, vp, vp]
+    lib.nbos_place_batch_host_wait.argtypes = [vp]
     lib.nbos_place_batch_noalloc.argtypes = [vp, vp, i64, vp, vp, vp, ctypes.c_int32]
     lib.nbos_select_executors.argtypes = [P(nbos_cluster_state), vp, vp, i64, vp, vp, vp]
     lib.nbos_cluster_sums.argtypes = [vp, vp, vp] + [ctypes.c_int32] * 4 + [vp, vp]
@@ -331,8 +334,7 @@ def nbos_place_batch_ex(snap, requests, out_hosts, out_found=None, stream=None, 
     nbos_place_batch(snap, requests, out_hosts, out_found, stream, config)
 
 
-def nbos_place_batch_host(snap: Snapshot, requests, out_hosts, out_found=None, stream=None) -> None:
-    """CPU tensors (pinned or not). Returns when the results are in `out_hosts` / `out_found`."""
+def _place_batch_host(name, snap, requests, out_hosts, out_found, stream):
     lib = load_library()
     _i32(requests, "requests", "cpu")
     _i32(out_hosts, "out_hosts", "cpu")
@@ -343,8 +345,25 @@ def nbos_place_batch_host(snap: Snapshot, requests, out_hosts, out_found=None, s
         raise ValueError("out_hosts must hold n_snapshots * batch * 3 values")
     if out_found is not None and out_found.numel() != snap.n_snapshots * b:
         raise ValueError("out_found must hold n_snapshots * batch values")
-    _check(lib.nbos_place_batch_host(snap.handle, _ptr(requests), b, _ptr(out_hosts),
-                                     _ptr(out_found), _stream_ptr(stream)))
+    _check(getattr(lib, name)(snap.handle, _ptr(requests), b, _ptr(out_hosts), _ptr(out_found),
+                              _stream_ptr(stream)))
+
+
+def nbos_place_batch_host(snap: Snapshot, requests, out_hosts, out_found=None, stream=None) -> None:
+    """CPU tensors (pinned or not). Returns when the results are in `out_hosts` / `out_found`."""
+    _place_batch_host("nbos_place_batch_host", snap, requests, out_hosts, out_found, stream)
+
+
+def nbos_place_batch_host_async(snap: Snapshot, requests, out_hosts, out_found=None, stream=None) -> None:
+    """CPU tensors (pinned, or the copies block). Returns once the work is queued; the results
+    are in `out_hosts` / `out_found` after nbos_place_batch_host_wait. The caller keeps the three
+    tensors alive and unchanged until then."""
+    _place_batch_host("nbos_place_batch_host_async", snap, requests, out_hosts, out_found, stream)
+
+
+def nbos_place_batch_host_wait(snap: Snapshot) -> None:
+    """Blocks until every host-buffer call made so far on the snapshot's device has delivered."""
+    _check(load_library().nbos_place_batch_host_wait(snap.handle))
 
 
 def nbos_place_batch_noalloc(snap: Snapshot, requests, out_hosts, out_found=None, stream=None,

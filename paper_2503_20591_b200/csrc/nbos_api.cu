@@ -80,22 +80,30 @@ int check_device(int *device, int *sm_count)
     return NBOS_OK;
 }
 
-// Side streams and events used by nbos_place_batch_host, one set per device, created on first use.
+// Streams, events and device staging used by the host-buffer entry points, per device, created on
+// first use: one stream for the copies in, one for the kernels, one for the copies out (each kind
+// of work is serial on the hardware anyway), and two sets of staging buffers taken in turn by
+// successive calls, so that the copies in of one call run beside the kernels of the call before
+// it and the copies out of the one before that.
 struct HostPipe {
-    static constexpr int kStreams = 3;
+    static constexpr int kSets = 2, kMaxChunks = 4;
     std::mutex mutex;
     bool ready = false;
-    cudaStream_t streams[kStreams] = {};
-    cudaEvent_t start = nullptr, done[kStreams] = {};
-    // The library's own stream-ordered pool for staging buffers. Its release threshold is
+    cudaStream_t s_in = nullptr, s_kernel = nullptr, s_out = nullptr;
+    cudaEvent_t start = nullptr;
+    cudaEvent_t h2d_done[kSets][kMaxChunks] = {}, kernel_done[kSets][kMaxChunks] = {};
+    cudaEvent_t kernels_done[kSets] = {};   // the last kernel that reads / writes the set's staging
+    cudaEvent_t out_done[kSets] = {};       // the last copy out of the set's staging
+    bool set_used[kSets] = {};
+    unsigned int turn = 0;
+    // The library's own stream-ordered pool for temporaries. Its release threshold is
     // unlimited, so the buffers of one call are reused by the next instead of going back to the
     // driver at every synchronisation (which costs more than the placement itself).
     cudaMemPool_t pool = nullptr;
-    // Device staging of nbos_place_batch_host (requests in, results out), kept between calls and
-    // grown when a larger batch comes: calls on a device take turns and each ends synchronised,
-    // so the buffer is free again when the next call starts.
-    char *stage = nullptr;
-    size_t stage_bytes = 0;
+    // Device staging (requests in, results out) of each set, kept between calls and grown when a
+    // larger batch comes.
+    char *stage[kSets] = {};
+    size_t stage_bytes[kSets] = {};
 };
 HostPipe g_pipes[64];
 std::mutex g_pipes_mutex;
@@ -106,9 +114,16 @@ int host_pipe(int device, HostPipe **out)
     std::lock_guard<std::mutex> lock(g_pipes_mutex);
     HostPipe &p = g_pipes[device];
     if (!p.ready) {
-        for (int j = 0; j < HostPipe::kStreams; ++j) {
-            NBOS_CUDA_TRY(cudaStreamCreateWithFlags(&p.streams[j], cudaStreamNonBlocking));
-            NBOS_CUDA_TRY(cudaEventCreateWithFlags(&p.done[j], cudaEventDisableTiming));
+        NBOS_CUDA_TRY(cudaStreamCreateWithFlags(&p.s_in, cudaStreamNonBlocking));
+        NBOS_CUDA_TRY(cudaStreamCreateWithFlags(&p.s_kernel, cudaStreamNonBlocking));
+        NBOS_CUDA_TRY(cudaStreamCreateWithFlags(&p.s_out, cudaStreamNonBlocking));
+        for (int k = 0; k < HostPipe::kSets; ++k) {
+            for (int c = 0; c < HostPipe::kMaxChunks; ++c) {
+                NBOS_CUDA_TRY(cudaEventCreateWithFlags(&p.h2d_done[k][c], cudaEventDisableTiming));
+                NBOS_CUDA_TRY(cudaEventCreateWithFlags(&p.kernel_done[k][c], cudaEventDisableTiming));
+            }
+            NBOS_CUDA_TRY(cudaEventCreateWithFlags(&p.kernels_done[k], cudaEventDisableTiming));
+            NBOS_CUDA_TRY(cudaEventCreateWithFlags(&p.out_done[k], cudaEventDisableTiming));
         }
         NBOS_CUDA_TRY(cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming));
         cudaMemPoolProps props = {};
@@ -389,9 +404,10 @@ int nbos_place_batch(const nbos_snapshot *snap, const int32_t *requests, int64_t
                                nullptr);
 }
 
-int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_host,
-                          int64_t batch_per_snapshot, int32_t *out_hosts_host,
-                          int32_t *out_found_host, void *cuda_stream)
+namespace {
+
+int place_batch_host(const nbos_snapshot *snap, const int32_t *requests_host, int64_t batch_per_snapshot,
+                     int32_t *out_hosts_host, int32_t *out_found_host, void *cuda_stream, bool synchronise)
 {
     if (!snap) return fail(NBOS_ERR_INVALID_ARG, "snapshot is NULL");
     if (batch_per_snapshot < 0 || batch_per_snapshot > ((int64_t)1 << 40) / snap->N)
@@ -406,74 +422,113 @@ int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_hos
                  found_bytes = out_found_host ? (size_t)total * 4 : 0;
     auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
 
-    // side streams for the copy / compute overlap, created once per process and device
     HostPipe *pipe = nullptr;
     int rc = host_pipe(snap->device, &pipe);
     if (rc) return rc;
     std::lock_guard<std::mutex> lock(pipe->mutex);
+    const int set = (int)(pipe->turn++ % HostPipe::kSets);
 
     const size_t need = up(req_bytes) + up(out_bytes) + up(found_bytes);
-    if (pipe->stage_bytes < need) {
-        if (pipe->stage) cudaFree(pipe->stage);
-        pipe->stage = nullptr;
-        pipe->stage_bytes = 0;
-        cudaError_t ea = cudaMalloc(reinterpret_cast<void **>(&pipe->stage), need);
+    if (pipe->stage_bytes[set] < need) {
+        // the call that used this set last may still be running: wait for it before the buffer goes
+        if (pipe->set_used[set]) NBOS_CUDA_TRY(cudaEventSynchronize(pipe->out_done[set]));
+        if (pipe->stage[set]) cudaFree(pipe->stage[set]);
+        pipe->stage[set] = nullptr;
+        pipe->stage_bytes[set] = 0;
+        cudaError_t ea = cudaMalloc(reinterpret_cast<void **>(&pipe->stage[set]), need);
         if (ea != cudaSuccess) {
             cudaGetLastError();
             return fail(NBOS_ERR_NO_MEMORY, "device staging allocation of %zu bytes failed: %s", need, cudaGetErrorString(ea));
         }
-        pipe->stage_bytes = need;
+        pipe->stage_bytes[set] = need;
     }
-    char *buf = pipe->stage;
+    char *buf = pipe->stage[set];
     int32_t *d_req = reinterpret_cast<int32_t *>(buf);
     int32_t *d_out = reinterpret_cast<int32_t *>(buf + up(req_bytes));
     int32_t *d_found = out_found_host ? reinterpret_cast<int32_t *>(buf + up(req_bytes) + up(out_bytes)) : nullptr;
 
-    // chunks of the flattened request list: copy in, place, copy out, round-robin over the side
-    // streams so that the copies of one chunk overlap the kernel of another. A chunk carries at
-    // least 2^30 (request, host) pairs: smaller launches lose more in kernel efficiency than the
-    // finer overlap gains (measured with 2, 4, 8, 16 and 32 chunks of the largest benchmark
-    // shape: 0.73, 0.68, 0.69, 0.78, 1.03 ms per call); at most four chunks. Every chunk launch
-    // plans itself. The copies in do not depend on anything queued on the caller's stream (the
-    // staging buffer is this call's alone) and start at once; only the kernels wait for it,
-    // because the snapshot may still be in the making there.
+    // Chunks of the flattened request list: copy in, place, copy out. A chunk carries at least
+    // 2^30 (request, host) pairs: smaller launches lose more in kernel efficiency than the finer
+    // overlap gains (measured with 2, 4, 8, 16 and 32 chunks of the largest benchmark shape);
+    // at most four chunks. Every chunk launch plans itself. The copies in depend on nothing
+    // queued on the caller's stream and start as soon as the set's request buffer is free (the
+    // kernels of the call that used it last have finished); only the kernels wait for the caller's
+    // stream, because the snapshot may still be in the making there; and the caller's stream in
+    // turn waits for the kernels (not for the copies out), so that a later snapshot update does
+    // not overtake them.
     const long long pairs = total * (long long)snap->Hpad;
     long long n_chunks = pairs >> 30;
     if (n_chunks < 1) n_chunks = 1;
-    if (n_chunks > 4) n_chunks = 4;
+    if (n_chunks > HostPipe::kMaxChunks) n_chunks = HostPipe::kMaxChunks;
     const long long chunk = (((total + n_chunks - 1) / n_chunks) + 31) & ~31ll;
     cudaError_t e = cudaEventRecord(pipe->start, stream);
-    bool waited[HostPipe::kStreams] = {};
-    int used = 0;
-    for (long long lo = 0, i = 0; lo < total && e == cudaSuccess && rc == NBOS_OK; lo += chunk, ++i) {
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(pipe->s_kernel, pipe->start, 0);
+    if (e == cudaSuccess && pipe->set_used[set]) {
+        e = cudaStreamWaitEvent(pipe->s_in, pipe->kernels_done[set], 0);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(pipe->s_kernel, pipe->out_done[set], 0);
+    }
+    for (long long lo = 0, c = 0; lo < total && e == cudaSuccess && rc == NBOS_OK; lo += chunk, ++c) {
         const long long n = total - lo < chunk ? total - lo : chunk;
-        const int j = (int)(i % HostPipe::kStreams);
-        cudaStream_t st = pipe->streams[j];
-        if (i < HostPipe::kStreams) used = (int)i + 1;
-        e = cudaMemcpyAsync(d_req + lo * 4, requests_host + lo * 4, (size_t)n * 16, cudaMemcpyHostToDevice, st);
+        e = cudaMemcpyAsync(d_req + lo * 4, requests_host + lo * 4, (size_t)n * 16, cudaMemcpyHostToDevice, pipe->s_in);
+        if (e == cudaSuccess) e = cudaEventRecord(pipe->h2d_done[set][c], pipe->s_in);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(pipe->s_kernel, pipe->h2d_done[set][c], 0);
         if (e != cudaSuccess) break;
-        if (!waited[j]) {
-            e = cudaStreamWaitEvent(st, pipe->start, 0);
-            if (e != cudaSuccess) break;
-            waited[j] = true;
-        }
-        rc = launch_place(snap, d_req, batch_per_snapshot, d_out, d_found, st, nullptr, lo, n);
+        rc = launch_place(snap, d_req, batch_per_snapshot, d_out, d_found, pipe->s_kernel, nullptr, lo, n);
         if (rc) break;
-        e = cudaMemcpyAsync(out_hosts_host + lo * 3, d_out + lo * 3, (size_t)n * 12, cudaMemcpyDeviceToHost, st);
+        e = cudaEventRecord(pipe->kernel_done[set][c], pipe->s_kernel);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(pipe->s_out, pipe->kernel_done[set][c], 0);
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(out_hosts_host + lo * 3, d_out + lo * 3, (size_t)n * 12, cudaMemcpyDeviceToHost, pipe->s_out);
         if (e == cudaSuccess && d_found)
-            e = cudaMemcpyAsync(out_found_host + lo, d_found + lo, (size_t)n * 4, cudaMemcpyDeviceToHost, st);
+            e = cudaMemcpyAsync(out_found_host + lo, d_found + lo, (size_t)n * 4, cudaMemcpyDeviceToHost, pipe->s_out);
     }
-    // join the side streams back into the caller's stream (also on the error paths, so that
-    // nothing of this call is still queued when the next one reuses the staging buffer)
-    for (int j = 0; j < used; ++j) {
-        cudaError_t e3 = cudaEventRecord(pipe->done[j], pipe->streams[j]);
-        if (e3 == cudaSuccess) e3 = cudaStreamWaitEvent(stream, pipe->done[j], 0);
-        if (e3 != cudaSuccess && e == cudaSuccess) e = e3;
+    // what was queued is accounted for also on the error paths, so that the set can be taken again
+    cudaError_t e3 = cudaEventRecord(pipe->kernels_done[set], pipe->s_kernel);
+    if (e3 == cudaSuccess) e3 = cudaStreamWaitEvent(stream, pipe->kernels_done[set], 0);
+    if (e3 == cudaSuccess) e3 = cudaStreamWaitEvent(pipe->s_out, pipe->kernels_done[set], 0);
+    if (e3 == cudaSuccess) e3 = cudaEventRecord(pipe->out_done[set], pipe->s_out);
+    if (e3 == cudaSuccess) pipe->set_used[set] = true;
+    const bool failed = rc != NBOS_OK || e != cudaSuccess || e3 != cudaSuccess;
+    cudaError_t e2 = cudaSuccess;
+    if (failed) {
+        cudaStreamSynchronize(pipe->s_in);
+        cudaStreamSynchronize(pipe->s_kernel);
+        cudaStreamSynchronize(pipe->s_out);
+    } else if (synchronise) {
+        e2 = cudaEventSynchronize(pipe->out_done[set]);
     }
-    cudaError_t e2 = cudaStreamSynchronize(stream);
     if (rc) return rc;
     if (e != cudaSuccess) return cuda_fail(e, "host <-> device copy");
-    if (e2 != cudaSuccess) return cuda_fail(e2, "cudaStreamSynchronize");
+    if (e3 != cudaSuccess) return cuda_fail(e3, "cudaEventRecord");
+    if (e2 != cudaSuccess) return cuda_fail(e2, "cudaEventSynchronize");
+    return NBOS_OK;
+}
+
+}  // namespace
+
+int nbos_place_batch_host(const nbos_snapshot *snap, const int32_t *requests_host,
+                          int64_t batch_per_snapshot, int32_t *out_hosts_host,
+                          int32_t *out_found_host, void *cuda_stream)
+{
+    return place_batch_host(snap, requests_host, batch_per_snapshot, out_hosts_host, out_found_host, cuda_stream, true);
+}
+
+int nbos_place_batch_host_async(const nbos_snapshot *snap, const int32_t *requests_host,
+                                int64_t batch_per_snapshot, int32_t *out_hosts_host,
+                                int32_t *out_found_host, void *cuda_stream)
+{
+    return place_batch_host(snap, requests_host, batch_per_snapshot, out_hosts_host, out_found_host, cuda_stream, false);
+}
+
+int nbos_place_batch_host_wait(const nbos_snapshot *snap)
+{
+    if (!snap) return fail(NBOS_ERR_INVALID_ARG, "snapshot is NULL");
+    HostPipe *pipe = nullptr;
+    int rc = host_pipe(snap->device, &pipe);
+    if (rc) return rc;
+    std::lock_guard<std::mutex> lock(pipe->mutex);
+    for (int k = 0; k < HostPipe::kSets; ++k)
+        if (pipe->set_used[k]) NBOS_CUDA_TRY(cudaEventSynchronize(pipe->out_done[k]));
     return NBOS_OK;
 }
 

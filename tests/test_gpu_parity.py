@@ -489,6 +489,44 @@ def test_host_buffer_entry_points(nb):
     nb.nbos_snapshot_destroy(s)
 
 
+def test_asynchronous_host_calls_in_a_row(nb):
+    """Six calls queued without waiting, batches of different sizes (the two staging sets grow and
+    are reused; the large ones go through in two chunks), a snapshot refresh between two of them,
+    pinned and pageable buffers; every call's results are checked after one wait at the end."""
+    import torch
+    stream = torch.cuda.Stream()
+    w = W.make_config(2, batch=2_200_000)
+    ref = oracle.place_workload(w, threads=CPU_THREADS)
+    lim = (torch.from_numpy(w.limit_num), torch.from_numpy(w.limit_den))
+    arrays = [torch.from_numpy(getattr(w, k)).reshape(-1).pin_memory() for k in w.HOST_FIELDS]
+    s = nb.nbos_snapshot_create_host(w.n_snapshots, w.n_hosts, *lim, *arrays, stream=stream)
+    sizes = [2_199_000, 5, 1_100_000, 2_200_000, 64, 2_100_001]
+    calls = []
+    for i, b in enumerate(sizes):
+        lo = 0 if b == w.batch else 7 * i
+        req = torch.from_numpy(np.ascontiguousarray(w.requests[:, lo: lo + b])).clone()
+        out = torch.full((1, b, 3), -9, dtype=torch.int32)
+        found = torch.full((1, b), -9, dtype=torch.int32)
+        if i != 4:
+            req, out, found = req.pin_memory(), out.pin_memory(), found.pin_memory()
+        if i == 3:
+            nb.nbos_snapshot_update_host(s, *lim, *arrays, stream=stream)
+        nb.nbos_place_batch_host_async(s, req, out, found if i % 2 == 0 else None, stream=stream)
+        calls.append((i, lo, b, req, out, found))
+    nb.nbos_place_batch_host_wait(s)
+    assert nb.nbos_snapshot_status(s) == nb.NBOS_OK
+    for i, lo, b, req, out, found in calls:
+        np.testing.assert_array_equal(out.numpy()[0], ref[0][0, lo: lo + b], err_msg=f"call {i}")
+        if i % 2 == 0:
+            np.testing.assert_array_equal(found.numpy()[0], ref[1][0, lo: lo + b], err_msg=f"call {i}")
+    # the blocking form takes its turn among them
+    req = torch.from_numpy(np.ascontiguousarray(w.requests[:, :1000])).pin_memory()
+    out = torch.empty((1, 1000, 3), dtype=torch.int32).pin_memory()
+    nb.nbos_place_batch_host(s, req, out, stream=stream)
+    np.testing.assert_array_equal(out.numpy()[0], ref[0][0, :1000])
+    nb.nbos_snapshot_destroy(s)
+
+
 def test_create_rejects_bad_values(nb):
     import torch
     w = W.make_config(0)
