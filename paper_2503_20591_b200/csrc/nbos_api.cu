@@ -104,6 +104,14 @@ struct HostPipe {
     // larger batch comes.
     char *stage[kSets] = {};
     size_t stage_bytes[kSets] = {};
+    // Device staging of the cluster-state arrays of nbos_snapshot_update_host, also two sets:
+    // they are copied on the copy-in stream, in call order with the request copies (a copy
+    // queued on another stream would wait behind whatever bulk copies are already running).
+    char *state_stage[kSets] = {};
+    size_t state_bytes[kSets] = {};
+    cudaEvent_t state_in[kSets] = {}, state_consumed[kSets] = {};
+    bool state_used[kSets] = {};
+    unsigned int state_turn = 0;
 };
 HostPipe g_pipes[64];
 std::mutex g_pipes_mutex;
@@ -124,6 +132,8 @@ int host_pipe(int device, HostPipe **out)
             }
             NBOS_CUDA_TRY(cudaEventCreateWithFlags(&p.kernels_done[k], cudaEventDisableTiming));
             NBOS_CUDA_TRY(cudaEventCreateWithFlags(&p.out_done[k], cudaEventDisableTiming));
+            NBOS_CUDA_TRY(cudaEventCreateWithFlags(&p.state_in[k], cudaEventDisableTiming));
+            NBOS_CUDA_TRY(cudaEventCreateWithFlags(&p.state_consumed[k], cudaEventDisableTiming));
         }
         NBOS_CUDA_TRY(cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming));
         cudaMemPoolProps props = {};
@@ -323,22 +333,36 @@ int nbos_snapshot_update_host(nbos_snapshot *snap, const nbos_snapshot_desc *des
     if (rc) return rc;
     const size_t cells = (size_t)snap->N * snap->H;
     const size_t arr_bytes = (cells * sizeof(int32_t) + 255) & ~(size_t)255;
-    void *staging = nullptr;
-    cudaError_t e = cudaMallocFromPoolAsync(&staging, 6 * arr_bytes, pipe->pool, stream);
-    if (e != cudaSuccess) {
-        cudaGetLastError();
-        return fail(NBOS_ERR_NO_MEMORY, "device allocation failed: %s", cudaGetErrorString(e));
+    std::lock_guard<std::mutex> lock(pipe->mutex);
+    const int k = (int)(pipe->state_turn++ % HostPipe::kSets);
+    if (pipe->state_bytes[k] < 6 * arr_bytes) {
+        // the update that used this set last may still be reading it
+        if (pipe->state_used[k]) NBOS_CUDA_TRY(cudaEventSynchronize(pipe->state_consumed[k]));
+        if (pipe->state_stage[k]) cudaFree(pipe->state_stage[k]);
+        pipe->state_stage[k] = nullptr;
+        pipe->state_bytes[k] = 0;
+        cudaError_t ea = cudaMalloc(reinterpret_cast<void **>(&pipe->state_stage[k]), 6 * arr_bytes);
+        if (ea != cudaSuccess) {
+            cudaGetLastError();
+            return fail(NBOS_ERR_NO_MEMORY, "device allocation failed: %s", cudaGetErrorString(ea));
+        }
+        pipe->state_bytes[k] = 6 * arr_bytes;
     }
+    char *staging = pipe->state_stage[k];
     const int32_t *src[6] = {desc->gpus_total, desc->gpus_subscribed, desc->gpus_committed,
                              desc->vram_gb, desc->millicpus, desc->mem_mb};
     const int32_t *dev[6];
+    cudaError_t e = pipe->state_used[k] ? cudaStreamWaitEvent(pipe->s_in, pipe->state_consumed[k], 0) : cudaSuccess;
     for (int i = 0; i < 6 && e == cudaSuccess; ++i) {
-        dev[i] = reinterpret_cast<const int32_t *>(static_cast<char *>(staging) + i * arr_bytes);
-        e = cudaMemcpyAsync(const_cast<int32_t *>(dev[i]), src[i], cells * sizeof(int32_t), cudaMemcpyHostToDevice, stream);
+        dev[i] = reinterpret_cast<const int32_t *>(staging + i * arr_bytes);
+        e = cudaMemcpyAsync(const_cast<int32_t *>(dev[i]), src[i], cells * sizeof(int32_t), cudaMemcpyHostToDevice, pipe->s_in);
     }
+    if (e == cudaSuccess) e = cudaEventRecord(pipe->state_in[k], pipe->s_in);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, pipe->state_in[k], 0);
     rc = e == cudaSuccess ? update_snapshot(snap, desc, dev[0], dev[1], dev[2], dev[3], dev[4], dev[5], stream)
                           : cuda_fail(e, "copying host-state arrays to the device");
-    cudaFreeAsync(staging, stream);
+    // also after an error: whatever was queued on `stream` comes before the set is written again
+    if (cudaEventRecord(pipe->state_consumed[k], stream) == cudaSuccess) pipe->state_used[k] = true;
     snap->owner_stream = stream;
     return rc;
 }
@@ -406,6 +430,10 @@ int nbos_place_batch(const nbos_snapshot *snap, const int32_t *requests, int64_t
 
 namespace {
 
+// chunks of an asynchronous call (measured at the largest benchmark shape, calls in a row with a
+// snapshot refresh between them: 1 / 2 / 3 / 4 chunks -> 0.53 / 0.44 / 0.51 / 0.52 ms per call)
+constexpr long long kAsyncChunks = 2;
+
 int place_batch_host(const nbos_snapshot *snap, const int32_t *requests_host, int64_t batch_per_snapshot,
                      int32_t *out_hosts_host, int32_t *out_found_host, void *cuda_stream, bool synchronise)
 {
@@ -460,6 +488,9 @@ int place_batch_host(const nbos_snapshot *snap, const int32_t *requests_host, in
     long long n_chunks = pairs >> 30;
     if (n_chunks < 1) n_chunks = 1;
     if (n_chunks > HostPipe::kMaxChunks) n_chunks = HostPipe::kMaxChunks;
+    // calls in a row have their requests on the device before their kernels' turn comes: fewer,
+    // larger launches then
+    if (!synchronise && n_chunks > kAsyncChunks) n_chunks = kAsyncChunks;
     const long long chunk = (((total + n_chunks - 1) / n_chunks) + 31) & ~31ll;
     cudaError_t e = cudaEventRecord(pipe->start, stream);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(pipe->s_kernel, pipe->start, 0);
