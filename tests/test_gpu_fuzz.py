@@ -3,6 +3,7 @@ flags and launch shapes, each compared bit for bit with the CPU checker."""
 from __future__ import annotations
 
 import dataclasses
+import os
 
 import numpy as np
 import pytest
@@ -49,7 +50,8 @@ def random_workload(rng) -> W.Workload:
         requests=np.ascontiguousarray(req.astype(np.int32)))
 
 
-@pytest.mark.parametrize("seed", range(150))
+# NBOS_FUZZ_CASES widens the campaign (e.g. 20000 for a long run; the default keeps the suite short)
+@pytest.mark.parametrize("seed", range(int(os.environ.get("NBOS_FUZZ_CASES", "150"))))
 def test_random_cases(nb, seed):
     rng = np.random.default_rng(10_000 + seed)
     w = random_workload(rng)
