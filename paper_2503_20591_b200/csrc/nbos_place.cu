@@ -1338,7 +1338,10 @@ int make_plan(const nbos_snapshot *s, long long total, long long batch, const nb
                     const long long on_sm = (blocks + s->sm_count - 1) / s->sm_count;
                     const int resident = (int)(on_sm < j ? on_sm : j);
                     const double cost = (double)on_sm * instr_block / issue_rate[resident > 4 ? 3 : resident - 1];
-                    if (!have || cost < best * 0.99) {
+                    // candidates come with the most resident blocks first; a later one must be
+                    // clearly cheaper (the estimate is good to a few per cent, and more resident
+                    // warps hide the second-level and exact work of sparse workloads better)
+                    if (!have || cost < best * 0.97) {
                         have = true;
                         best = cost;
                         L = cand;
