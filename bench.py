@@ -228,7 +228,7 @@ def time_launches(torch, stream, fn, reps: int, warm: int = 3):
 
 
 def workload_character(w, hosts: np.ndarray, found: np.ndarray, sample: int = 1024):
-    """What the inputs and outputs look like, so that a reader can judge how much the pair
+    """What the inputs and outputs look like, so that a reader can tell how much the pair
     evaluation has to do: how many hosts each request found, how many different answers the
     batch has, how often each test of Sections 3.2.1 / 3.4.1 rejects a (request, host) pair
     (sampled requests x all hosts, every test counted on its own), and how far into the key order
