@@ -211,10 +211,13 @@ int nbos_snapshot_create_host(const nbos_snapshot_desc *desc, void *cuda_stream,
  * The caller must make sure that no placement on ANOTHER stream is still using the snapshot;
  * work queued earlier on the same stream is ordered before the update.
  *   nbos_snapshot_update       arrays are DEVICE memory (16-byte aligned), read by the queued work
- *   nbos_snapshot_update_host  arrays are HOST memory; staged through the library's memory pool.
+ *   nbos_snapshot_update_host  arrays are HOST memory; copied into device staging the library
+ *                              keeps per device (two sets, taken in turn) on its copy-in stream,
+ *                              in call order with the request copies of the host-buffer placement
+ *                              calls; the derivation queued on `cuda_stream` waits for the copies.
  *                              Pageable arrays have been read when the call returns; PINNED arrays
- *                              are read asynchronously by copies queued on `cuda_stream`: keep
- *                              them unchanged until that work has finished.
+ *                              are read asynchronously: keep them unchanged until `cuda_stream`
+ *                              has reached the end of the update.
  * Errors at call time: INVALID_ARG (shape / flags differ, NULL or misaligned pointers, bad limit),
  * NO_MEMORY, CUDA.
  */
