@@ -527,6 +527,64 @@ def test_asynchronous_host_calls_in_a_row(nb):
     nb.nbos_snapshot_destroy(s)
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_random_sequences_of_host_calls(nb, seed):
+    """Refreshes from three different states, asynchronous and blocking placements of random sizes
+    and waits, in random order on one stream; every placement is checked against the state that
+    was current when it was queued."""
+    import torch
+    rng = np.random.default_rng(seed)
+    hosts, pool = int(rng.choice([33, 700, 1024])), int(rng.choice([5000, 120_000]))
+    states = [W.uniform_cluster(hosts, pool, seed=seed * 7 + k) for k in range(3)]
+    w0 = states[0]
+    stream = torch.cuda.Stream() if seed % 2 else torch.cuda.current_stream()
+
+    def pin(a):
+        return torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+
+    lim = (torch.from_numpy(w0.limit_num), torch.from_numpy(w0.limit_den))
+    arrs = [[pin(getattr(s, k).reshape(-1)) for k in s.HOST_FIELDS] for s in states]
+    snap = nb.nbos_snapshot_create_host(1, hosts, *lim, *arrs[0], stream=stream)
+    cur, pending = 0, []
+
+    def check_all():
+        for si, lo, b, req, out, found in pending:
+            s = states[si]
+            ref = oracle.place(*[getattr(s, k)[0] for k in s.HOST_FIELDS], int(s.limit_num[0]), int(s.limit_den[0]),
+                               w0.requests[0, lo:lo + b], replicas_R=s.replicas_R)
+            np.testing.assert_array_equal(out.numpy()[0], ref[0], err_msg=f"state {si}, requests {lo}..{lo + b}")
+            np.testing.assert_array_equal(found.numpy()[0], ref[1])
+        pending.clear()
+
+    for _ in range(int(rng.integers(6, 14))):
+        op = rng.choice(["update", "async", "async", "async", "block", "wait"])
+        if op == "update":
+            cur = int(rng.integers(0, 3))
+            nb.nbos_snapshot_update_host(snap, *lim, *arrs[cur], stream=stream)
+        elif op == "wait":
+            nb.nbos_place_batch_host_wait(snap)
+            check_all()
+        else:
+            b = int(rng.choice([1, 31, 1000, 4097]))
+            lo = int(rng.integers(0, pool - b + 1))
+            req = pin(w0.requests[:, lo:lo + b]) if rng.random() < 0.8 else torch.from_numpy(np.ascontiguousarray(w0.requests[:, lo:lo + b]))
+            out, found = torch.full((1, b, 3), -9, dtype=torch.int32), torch.full((1, b), -9, dtype=torch.int32)
+            if rng.random() < 0.8:
+                out, found = out.pin_memory(), found.pin_memory()
+            if op == "async":
+                nb.nbos_place_batch_host_async(snap, req, out, found, stream=stream)
+                pending.append((cur, lo, b, req, out, found))
+            else:
+                nb.nbos_place_batch_host(snap, req, out, found, stream=stream)
+                pending.append((cur, lo, b, req, out, found))
+                check_all()
+    nb.nbos_place_batch_host_wait(snap)
+    check_all()
+    assert nb.nbos_snapshot_status(snap) == nb.NBOS_OK
+    torch.cuda.synchronize()
+    nb.nbos_snapshot_destroy(snap)
+
+
 def test_create_rejects_bad_values(nb):
     import torch
     w = W.make_config(0)
